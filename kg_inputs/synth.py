@@ -1,0 +1,161 @@
+"""Counter-based synthetic tensor generator (integer-exact, so host and device agree bit for bit).
+
+Element `i` of the tensor with id `tid` under seed `s` is a pure function of (s, tid, i):
+
+    base = splitmix64(splitmix64(s) + tid)            # one stream per tensor
+    u    = splitmix64(base + i)                        # 64 random bits per element
+    g    = (sum of the eight bytes of u) - 1020        # integer in [-1020, 1020], mean 0
+    x    = float32(g) * scale                          # ONE fp32 multiply, scale = std / GAUSS_INT_STD
+    (bf16 models)  x = round-to-nearest-even of x to bfloat16
+
+The byte sum is an Irwin-Hall(8) variable: bell shaped, variance 8*(256^2-1)/12 = 43690,
+support +-4.88 sigma.  Every intermediate is an exact integer below 2^24, the single
+multiply is IEEE fp32, and the bf16 rounding is bit arithmetic, so a C, numpy or CUDA
+implementation produces identical bits without sharing code.
+
+splitmix64 is the published 64-bit mixing function of Steele, Lea and Flood's SplitMix
+generator (golden-gamma increment followed by two xor-shift-multiply rounds).
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from enum import IntEnum
+
+import numpy as np
+
+_M64 = (1 << 64) - 1
+_GAMMA = 0x9E3779B97F4A7C15
+_C1 = 0xBF58476D1CE4E5B9
+_C2 = 0x94D049BB133111EB
+
+GAUSS_INT_VAR = 43690.0            # 8 * (256**2 - 1) / 12
+GAUSS_INT_STD = math.sqrt(GAUSS_INT_VAR)
+
+
+class TensorId(IntEnum):
+    """Stream ids. Per-layer tensors use LAYER_BASE + 16*layer + k; the adapter is layer index L."""
+    EMBED = 1
+    HEAD = 2
+    PROMPT = 3
+    HIDDEN = 4        # config-3 microbench hidden rows
+    GFINAL = 6        # gain of the target's final norm
+    LAYER_BASE = 100
+    # k within a layer
+    WQKV = 0
+    WO = 1
+    WGATE = 2
+    WUP = 3
+    WDOWN = 4
+    G1 = 5            # decoder layer: attention-input norm gain; adapter: input norm gain
+    G2 = 6            # decoder layer: FFN-input norm gain;       adapter: last norm gain
+    KCACHE = 8
+    VCACHE = 9
+
+
+def layer_tid(layer: int, k: int) -> int:
+    return int(TensorId.LAYER_BASE) + 16 * int(layer) + int(k)
+
+
+def splitmix64(z):
+    """splitmix64 of a Python int or of a numpy uint64 array (wrapping arithmetic)."""
+    if isinstance(z, (int, np.integer)):
+        z = (int(z) + _GAMMA) & _M64
+        z = ((z ^ (z >> 30)) * _C1) & _M64
+        z = ((z ^ (z >> 27)) * _C2) & _M64
+        return z ^ (z >> 31)
+    z = np.asarray(z, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        z = z + np.uint64(_GAMMA)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(_C1)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(_C2)
+        return z ^ (z >> np.uint64(31))
+
+
+def stream_base(seed: int, tid: int) -> int:
+    return splitmix64((splitmix64(int(seed) & _M64) + int(tid)) & _M64)
+
+
+def _u64_stream(seed: int, tid: int, start: int, count: int) -> np.ndarray:
+    base = stream_base(seed, tid)
+    idx = np.arange(start, start + count, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        return splitmix64(idx + np.uint64(base))
+
+
+def gauss_ints(seed: int, tid: int, start: int, count: int) -> np.ndarray:
+    """The integer g of elements [start, start+count) as int32."""
+    u = _u64_stream(seed, tid, start, count)
+    b = u.view(np.uint8).reshape(count, 8)
+    return b.sum(axis=1, dtype=np.int32) - np.int32(1020)
+
+
+def scale_f32(std: float) -> np.float32:
+    """The fp32 scale every implementation multiplies by (computed once, in double, then rounded)."""
+    return np.float32(float(std) / GAUSS_INT_STD)
+
+
+def gauss_f32(seed: int, tid: int, start: int, count: int, std: float) -> np.ndarray:
+    g = gauss_ints(seed, tid, start, count).astype(np.float32)
+    return g * scale_f32(std)
+
+
+def round_to_bf16_f32(x: np.ndarray) -> np.ndarray:
+    """Round fp32 to the nearest bfloat16 (ties to even), returned widened back to fp32."""
+    bits = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    lsb = (bits >> np.uint32(16)) & np.uint32(1)
+    with np.errstate(over="ignore"):
+        r = bits + np.uint32(0x7FFF) + lsb
+    r &= np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def uniform_tokens(seed: int, tid: int, count: int, vocab: int) -> np.ndarray:
+    u = _u64_stream(seed, tid, 0, count)
+    return (u % np.uint64(vocab)).astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------
+# Bulk host fill.  A small C routine (kg_inputs/fill.c, OpenMP) does the same computation
+# for multi-GB tensors; numpy is the reference and the fallback.
+# --------------------------------------------------------------------------------------
+_lib = None
+
+
+def _load_fill_lib():
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkg_inputs_fill.so")
+    if os.path.exists(path):
+        try:
+            lib = ctypes.CDLL(path)
+            lib.kgi_fill_f32.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                         ctypes.c_uint64, ctypes.c_float, ctypes.c_int]
+            lib.kgi_fill_f32.restype = None
+            _lib = lib
+        except OSError:
+            _lib = False
+    else:
+        _lib = False
+    return _lib
+
+
+def fill_f32(seed: int, tid: int, count: int, std: float, bf16: bool,
+             force_numpy: bool = False) -> np.ndarray:
+    """A whole tensor (flat, fp32 container).  With bf16=True every value is bf16-representable."""
+    lib = None if force_numpy else _load_fill_lib()
+    if lib:
+        out = np.empty(count, dtype=np.float32)
+        lib.kgi_fill_f32(out.ctypes.data, ctypes.c_uint64(stream_base(seed, tid)),
+                         ctypes.c_uint64(0), ctypes.c_uint64(count),
+                         ctypes.c_float(float(scale_f32(std))), 1 if bf16 else 0)
+        return out
+    out = np.empty(count, dtype=np.float32)
+    step = 1 << 22
+    for s in range(0, count, step):
+        n = min(step, count - s)
+        x = gauss_f32(seed, tid, s, n, std)
+        out[s:s + n] = round_to_bf16_f32(x) if bf16 else x
+    return out
