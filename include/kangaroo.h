@@ -1,0 +1,198 @@
+/* kangaroo.h - C ABI of the B200 (sm_100a) implementation of the Kangaroo batch-1
+ * self-speculative decode step (Liu et al., "Kangaroo: Lossless Self-Speculative Decoding
+ * via Double Early Exiting").
+ *
+ * The library owns no memory: the caller hands in one device arena and one CUDA stream, and
+ * every kernel runs on that stream.  No call allocates device memory or creates streams.
+ * All functions return KG_OK (0) or a negative kg_status; none throws or aborts.  Argument and
+ * state errors launch nothing.
+ *
+ * Pointer suffixes: _host = host memory, _dev = device memory on the current device.
+ *
+ * Model (Section 3.1, Figure 2 of the paper): target M^b = LLaMA-style decoder with L layers;
+ * self-draft model M^s = A o M^b[:l] (first l layers + adapter A = one attention with an input
+ * and a last RMS norm) re-using the target's LM head.  Matrices are row-major
+ * [out_features, in_features]; W_qkv is [3d, d] (q rows, then k rows, then v rows).
+ */
+#ifndef KANGAROO_H_
+#define KANGAROO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KG_M_MAX 16               /* most rows one pass may carry: gamma_max + 1 <= KG_M_MAX */
+#define KG_GAMMA_MAX (KG_M_MAX - 1)
+
+typedef enum {
+    KG_OK = 0,
+    KG_E_ARG = -1,       /* NULL pointer, bad size, unsupported shape */
+    KG_E_STATE = -2,     /* call order violated (e.g. kg_verify without a pending draft) */
+    KG_E_NOMEM = -3,     /* arena too small */
+    KG_E_SEQ_FULL = -4,  /* the sequence would exceed max_seq */
+    KG_E_CUDA = -5,      /* a CUDA runtime call failed */
+    KG_E_TIMEOUT = -6    /* a bounded device-side wait expired; the model must be re-initialised */
+} kg_status;
+
+enum { KG_F32 = 0, KG_BF16 = 1 };            /* storage type of weights and KV cache */
+enum { KG_STOP_KEEP = 0, KG_STOP_DROP = 1 }; /* is the draft whose confidence is <= eta kept? */
+
+typedef struct kg_model kg_model;            /* opaque host handle */
+
+typedef struct {
+    uint32_t struct_size;                    /* = sizeof(kg_config) */
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;   /* L, d, H, hd, F, V */
+    int32_t exit_layer;                      /* l, 1 <= l < L (Section 3.1) */
+    int32_t dtype;                           /* KG_F32 | KG_BF16 */
+    float rms_eps, rope_theta, logit_scale;  /* logits z = logit_scale * W_head y */
+    int32_t max_seq, page_size, gamma_max;   /* KV capacity in tokens; tokens per KV page; largest gamma */
+    int32_t debug_logits;                    /* 1: keep every computed logit row in HBM for kg_debug_logits */
+    int32_t page_shuffle;                    /* 1: non-identity page table (exercises the indirection) */
+    /* synthetic initialisation, used when kg_init_model gets weights == NULL */
+    uint64_t seed;
+    float init_std, embed_std, deep_resid_scale, adapter_resid_scale, gain_std;
+} kg_config;
+
+/* Borrowed device pointers to caller-provided weights (optional).  Arrays are HOST arrays of
+ * device pointers.  Index L (= n_layers) of wqkv / wo / g1 / g2 is the adapter (g1 = input norm
+ * gain, g2 = last norm gain).  Matrices have the model's storage dtype, gains are fp32. */
+typedef struct {
+    const void* embed_dev;                   /* [V, d] */
+    const void* head_dev;                    /* [V, d] */
+    const float* g_final_dev;                /* [d] */
+    const void* const* wqkv_dev;             /* L+1 x [3d, d] */
+    const void* const* wo_dev;               /* L+1 x [d, d] */
+    const void* const* wgate_dev;            /* L   x [F, d] */
+    const void* const* wup_dev;              /* L   x [F, d] */
+    const void* const* wdown_dev;            /* L   x [d, F] */
+    const float* const* g1_dev;              /* L+1 x [d] */
+    const float* const* g2_dev;              /* L+1 x [d] */
+} kg_weights;
+
+typedef struct {
+    int32_t n_drafted;                       /* n_d: drafts kept this round */
+    int32_t n_steps;                         /* adapter+head passes run (= confidences computed) */
+    int32_t tokens[KG_GAMMA_MAX];            /* x'_1 .. x'_{n_d} */
+    float conf[KG_GAMMA_MAX];                /* every confidence computed, a dropped token's included */
+} kg_draft_out;
+
+typedef struct {
+    int32_t n_rows;                          /* M = n_d + 1 rows verified */
+    int32_t n_accept;                        /* k: accepted drafts */
+    int32_t n_emitted;                       /* k + 1 */
+    int32_t emitted[KG_M_MAX];               /* x'_1..x'_k, t_k */
+    int32_t target[KG_M_MAX];                /* t_0 .. t_{n_d}: the target's greedy token per row */
+} kg_verify_out;
+
+typedef struct {
+    int32_t rounds;                          /* |S| */
+    int32_t tokens;                          /* sum of S (tokens produced by rounds; x_0 of prefill not counted) */
+    int32_t draft_steps;                     /* adapter+head passes in total */
+    int32_t drafted;                         /* drafts kept in total */
+    int32_t accepted;                        /* drafts accepted in total */
+    double cr;                               /* Eq. 1 */
+    double ctar[KG_M_MAX + 1];               /* Eq. 2 for w = 0 .. KG_M_MAX */
+    float ms_decode;                         /* device time of the decode loop (CUDA events), 0 if not measured */
+} kg_stats;
+
+/* Bytes of arena kg_init_model needs: KV pages, activations, scratch, and (own_weights != 0)
+ * the synthetic weights themselves.  Returns 0 on an invalid config. */
+size_t kg_workspace_bytes(const kg_config* cfg, int own_weights);
+
+/* Builds a model inside `arena_dev` (256-byte aligned, >= kg_workspace_bytes).  weights == NULL:
+ * fills seeded synthetic weights on the device with the counter-based generator (bit-identical
+ * to the host generator of the test inputs).  The arena and the stream stay owned by the caller
+ * and must outlive the model.  `cuda_stream` is a cudaStream_t. */
+int kg_init_model(const kg_config* cfg, const kg_weights* weights, void* arena_dev, size_t arena_bytes,
+                  void* cuda_stream, kg_model** out);
+int kg_free_model(kg_model* m);              /* frees the host handle only */
+
+/* Forget the sequence (KV lengths, round state); weights stay. */
+int kg_reset(kg_model* m);
+
+/* All L layers over the prompt, the adapter's K/V for every prompt position, and
+ * x_0 = argmax M^b(. | prompt) (Figure 2's starting point).  Requires a reset model.
+ * kg_prefill copies the prompt from the host; if first_token_host != NULL it synchronises the
+ * stream and returns x_0.  kg_prefill_device reads prompt ids already in device memory and
+ * never synchronises. */
+int kg_prefill(kg_model* m, const int32_t* prompt_host, int32_t n, int32_t* first_token_host);
+int kg_prefill_device(kg_model* m, const int32_t* prompt_dev, int32_t n);
+
+/* One round's draft phase (Section 3.2, Eq. 4; Figure 2): run M^s one token at a time from x_0,
+ * stop when the top-1 probability p <= eta or gamma tokens are drafted; the early features
+ * f_0..f_{n_d} stay on the device for kg_verify.  The whole loop, its exit test included, runs on
+ * the device.  out (nullable): copies the result and synchronises the stream. */
+int kg_draft(kg_model* m, float eta, int32_t gamma, int32_t stop_mode, kg_draft_out* out);
+
+/* Verify the pending unit [f_0..f_{n_d}] with layers l+1..L in one pass, accept the longest
+ * prefix of drafts that equals the target's greedy tokens, discard the rest, roll the KV caches
+ * back (Section 3; Figure 2).  out (nullable): copies the result and synchronises. */
+int kg_verify(kg_model* m, kg_verify_out* out);
+
+/* Device-resident decode loop: rounds of draft + verify + accept until at least max_new tokens
+ * (x_0 included) exist; one kernel launch, no host round-trip.  Requires a prefilled model.
+ * stats (nullable): synchronises and fills it. */
+int kg_decode(kg_model* m, int32_t max_new, float eta, int32_t gamma, int32_t stop_mode, kg_stats* stats);
+
+/* Plain greedy autoregressive decoding of the target (the definition Kangaroo must reproduce,
+ * Section 1): n_tokens tokens in total, x_0 included.  out_host (nullable) receives them. */
+int kg_decode_ar(kg_model* m, int32_t n_tokens, int32_t* out_host);
+
+/* reset + prefill + decode + read-back.  Returns exactly max_new tokens (x_0 first); the last
+ * round is truncated so that sum(S) counts only returned tokens (Section 3, list S). */
+int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_prompt, int32_t max_new,
+                float eta, int32_t gamma, int32_t stop_mode,
+                int32_t* out_tokens_host, int32_t* n_out, kg_stats* stats);
+
+/* Copies tokens produced so far (x_0 first) / the accepted-length list S to the host; synchronises. */
+int kg_read_tokens(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out);
+int kg_read_S(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out);
+
+/* Parity helpers (need cfg.debug_logits = 1).  which = 0: draft logits of step `row` of the last
+ * round; which = 1: verify / AR / prefill logits of row `row` of the last pass.  Copies V floats. */
+int kg_debug_logits(kg_model* m, int32_t which, int32_t row, float* out_host);
+
+/* Reads `count` elements starting at `offset` of a weight tensor, widened to fp32.
+ * name: "embed","head","wqkv","wo","wgate","wup","wdown","g1","g2","g_final"; layer = L for the adapter. */
+int kg_read_weight(kg_model* m, const char* name, int32_t layer, uint64_t offset, uint64_t count, float* out_host);
+
+/* Microbenchmark support (the verify-step / draft-step shapes of the evaluation): pretend the
+ * sequence has T tokens by filling every KV cache [0, T) with seeded N(0,1) entries, sets
+ * x_0 = token, and, if n_d >= 0, a pending draft of n_d seeded tokens with N(0,1) early features. */
+int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t seed);
+
+/* ---- single operators on caller buffers (unit tests and microbenchmarks) ------------------------
+ * All pointers are device pointers; `scratch_dev` must hold kg_op_scratch_bytes() bytes; the
+ * call is asynchronous on `cuda_stream`.  dtype is KG_F32 or KG_BF16 and is the type of W / KV. */
+size_t kg_op_scratch_bytes(void);
+
+/* out[M, N] = (resid ? resid : 0) + RMSNorm(x; gain, eps) W^T   (gain == NULL: no norm)
+ * swiglu != 0: W is W_gate, W2 is W_up (both [N, K]) and out = SiLU(gate) * up. */
+int kg_op_linear(int32_t dtype, const void* W_dev, const void* W2_dev, int32_t N, int32_t K,
+                 const float* x_dev, int32_t M, const float* gain_dev, float eps,
+                 const float* resid_dev, int32_t swiglu, float* out_dev,
+                 void* scratch_dev, void* cuda_stream);
+
+/* Fused LM head (Figure 2: shared head; Eq. 4's confidence): z = logit_scale * RMSNorm(x) W_head^T,
+ * per row the arg max (lowest index on ties) and p = 1 / sum_i exp(z_i - z_max).
+ * logits_dev (nullable) receives z [M, V]. */
+int kg_op_lm_head(int32_t dtype, const void* W_head_dev, int32_t V, int32_t K, const float* x_dev, int32_t M,
+                  const float* gain_dev, float eps, float logit_scale,
+                  int32_t* tok_dev, float* p_dev, float* logits_dev, void* scratch_dev, void* cuda_stream);
+
+/* Causal attention of M new rows at positions pos0.. over a paged KV cache (RoPE fused): takes the
+ * raw q,k,v rows qkv[M, 3d], rotates q and k, appends k and v to the cache pages, and returns
+ * out[M, d] = concat_heads softmax(q K^T / sqrt(hd)) V.  Cache layout: [page][head][slot][hd]. */
+int kg_op_attention(int32_t dtype, const float* qkv_dev, int32_t M, int32_t pos0, int32_t n_heads, int32_t head_dim,
+                    float rope_theta, void* kcache_dev, void* vcache_dev, const int32_t* page_table_dev,
+                    int32_t page_size, float* out_dev, void* scratch_dev, void* cuda_stream);
+
+const char* kg_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KANGAROO_H_ */

@@ -19,4 +19,4 @@ from .synth import (  # noqa: F401
     TensorId,
     GAUSS_INT_STD,
 )
-from .configs import KgShape, CONFIGS, get_config, make_weights, make_prompt, param_counts  # noqa: F401
+from .configs import KgShape, CONFIGS, get_config, make_weights, make_prompt, param_counts, microbench_state  # noqa: F401

@@ -93,15 +93,16 @@ def tensor_spec(shape: KgShape, name: str, layer: int | None = None):
     """(stream id, (rows, cols), std) of one weight matrix.  `layer` in [0, L) for decoder
     layers, layer == L for the adapter (which has only wqkv and wo)."""
     d, F, V, L = shape.d_model, shape.d_ffn, shape.vocab, shape.n_layers
-    s = shape.init_std
+    f32 = lambda v: float(np.float32(v))      # the C ABI carries these as fp32; products are formed in double
+    s = f32(shape.init_std)
     if name == "embed":
-        return int(TensorId.EMBED), (V, d), shape.embed_std
+        return int(TensorId.EMBED), (V, d), f32(shape.embed_std)
     if name == "head":
         return int(TensorId.HEAD), (V, d), s
     assert layer is not None
     is_adapter = layer == L
     deep = (not is_adapter) and layer >= shape.exit_layer
-    out_scale = shape.adapter_resid_scale if is_adapter else (shape.deep_resid_scale if deep else 1.0)
+    out_scale = f32(shape.adapter_resid_scale) if is_adapter else (f32(shape.deep_resid_scale) if deep else 1.0)
     if name == "wqkv":
         return layer_tid(layer, TensorId.WQKV), (3 * d, d), s
     if name == "wo":
@@ -125,7 +126,7 @@ def weight_tensor(shape: KgShape, name: str, layer: int | None = None, force_num
 def gain_vector(shape: KgShape, tid: int) -> np.ndarray:
     """Norm gain 1 + gain_std * g (fp32, never rounded to bf16); exactly 1 when gain_std == 0."""
     d = shape.d_model
-    g = synth.gauss_ints(shape.seed, tid, 0, d).astype(np.float32) * synth.scale_f32(shape.gain_std)
+    g = synth.gauss_ints(shape.seed, tid, 0, d).astype(np.float32) * synth.scale_f32(float(np.float32(shape.gain_std)))
     return (np.float32(1.0) + g).astype(np.float32)
 
 
@@ -157,3 +158,19 @@ def make_weights(shape: KgShape, force_numpy=False) -> dict:
 def make_prompt(shape: KgShape, n: int | None = None) -> np.ndarray:
     n = shape.n_prompt if n is None else n
     return synth.uniform_tokens(shape.seed, int(TensorId.PROMPT), n, shape.vocab)
+
+
+def microbench_state(shape: KgShape, T: int, n_d: int, seed: int) -> dict:
+    """Inputs of the verify-step / draft-step microbenchmark: every KV cache holds seeded N(0,1)
+    entries for positions [0, T) (rounded to the storage type), the early-feature slots hold
+    N(0,1) rows (slot 0 = position T-1, slot 1+j = f_j), plus x_0 and n_d draft token ids.
+    Element (pos, head, e) of a cache is element (pos*H + head)*hd + e of its stream."""
+    H, hd, d, L = shape.n_heads, shape.head_dim, shape.d_model, shape.n_layers
+    bf = shape.dtype == "bf16"
+    k, v = [], []
+    for i in range(L + 1):
+        k.append(synth.fill_f32(seed, layer_tid(i, TensorId.KCACHE), T * H * hd, 1.0, bf).reshape(T, H, hd))
+        v.append(synth.fill_f32(seed, layer_tid(i, TensorId.VCACHE), T * H * hd, 1.0, bf).reshape(T, H, hd))
+    feat = synth.fill_f32(seed, int(TensorId.HIDDEN), 17 * d, 1.0, False).reshape(17, d)
+    toks = synth.uniform_tokens(seed, int(TensorId.DRAFT), 1001, shape.vocab)
+    return {"k": k, "v": v, "feat": feat, "x0": int(toks[1000]), "drafts": [int(t) for t in toks[:max(n_d, 0)]]}

@@ -41,6 +41,7 @@ class TensorId(IntEnum):
     PROMPT = 3
     HIDDEN = 4        # config-3 microbench hidden rows
     GFINAL = 6        # gain of the target's final norm
+    DRAFT = 7         # microbenchmark token ids
     LAYER_BASE = 100
     # k within a layer
     WQKV = 0

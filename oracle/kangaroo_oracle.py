@@ -187,12 +187,12 @@ class KangarooOracle:
         return x @ W.T
 
     # -- blocks ------------------------------------------------------------------------
-    def attention(self, n, pos0, wqkv, wo, cache):
-        """Causal multi-head attention of the normalised rows n[M, d] at positions pos0.., appending
-        their K/V rows to `cache`.  Row i attends to keys 0 .. pos0+i.  Returns Wo . concat_heads(...)."""
-        M = n.shape[0]
+    def attention_core(self, qkv, pos0, cache):
+        """Causal multi-head attention given the raw rows qkv[M, 3d] = [q | k | v] at positions pos0..:
+        rotate q and k, append k and v to `cache`, row i attends to keys 0 .. pos0+i.
+        Returns concat_heads softmax(q K^T / sqrt(hd)) V, shape [M, d]."""
+        M = qkv.shape[0]
         d, H, hd = self.d, self.H, self.hd
-        qkv = self.linear(n, wqkv)
         out = np.zeros((M, d), self.dt)
         for i in range(M):
             pos = pos0 + i
@@ -205,7 +205,11 @@ class KangarooOracle:
             scores = np.einsum("hd,thd->ht", q, K) / np.sqrt(self.dt.type(hd))
             p = softmax_rows(scores)
             out[i] = np.einsum("ht,thd->hd", p, V).reshape(d)
-        return self.linear(out, wo)
+        return out
+
+    def attention(self, n, pos0, wqkv, wo, cache):
+        """Wo . Attn(n) for the normalised rows n[M, d] at positions pos0.., appending their K/V to `cache`."""
+        return self.linear(self.attention_core(self.linear(n, wqkv), pos0, cache), wo)
 
     def decoder_layer(self, h, pos0, i):
         """One LLaMA block: h += Wo Attn(RMSNorm(h)); h += Wdown(SiLU(Wgate n) * (Wup n))."""

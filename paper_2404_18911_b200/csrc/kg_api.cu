@@ -1,0 +1,792 @@
+// Host side of the C ABI declared in include/kangaroo.h: arena layout, synthetic weight fill,
+// launches of the persistent decode kernel, small result copies.  No device allocation anywhere.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/kangaroo.h"
+#include "kg_engine.cuh"
+
+using namespace kg;
+
+// ------------------------------------------------------------------------------------ generator
+// Counter-based generator, implemented here independently of the host-side test generator:
+//   base = mix(mix(seed) + tid); u = mix(base + i); g = bytesum(u) - 1020; x = float(g) * scale.
+// mix is the SplitMix64 output function (Steele, Lea, Flood).
+namespace {
+
+__host__ __device__ inline uint64_t mix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+inline uint64_t stream_base(uint64_t seed, uint64_t tid) { return mix64(mix64(seed) + tid); }
+inline float gen_scale(double std_) { return (float)(std_ / std::sqrt(43690.0)); }
+
+__device__ __forceinline__ float gen_value(uint64_t base, uint64_t i, float scale) {
+    const uint64_t u = mix64(base + i);
+    const unsigned lo = (unsigned)u, hi = (unsigned)(u >> 32);
+    // byte sum via two SIMD-in-register adds
+    const unsigned s2 = (lo & 0x00ff00ffu) + ((lo >> 8) & 0x00ff00ffu) + (hi & 0x00ff00ffu) + ((hi >> 8) & 0x00ff00ffu);
+    const int g = (int)((s2 & 0xffffu) + (s2 >> 16)) - 1020;
+    return __fmul_rn((float)g, scale);
+}
+
+template <typename WT>
+__global__ void fill_matrix_kernel(WT* out, uint64_t base, uint64_t count, float scale) {
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x)
+        out[i] = float_to_wt<WT>(gen_value(base, i, scale));
+}
+__global__ void fill_gain_kernel(float* out, uint64_t base, int count, float scale) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x)
+        out[i] = __fadd_rn(1.0f, gen_value(base, (uint64_t)i, scale));
+}
+__global__ void fill_f32_kernel(float* out, uint64_t base, uint64_t count, float scale) {
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x)
+        out[i] = gen_value(base, i, scale);
+}
+// KV cache entries for positions [0, T): element index (pos*H + head)*hd + e of the stream.
+template <typename WT>
+__global__ void fill_cache_kernel(WT* cache, const int* page_table, uint64_t base, int T, int H, int hd, int ps, float scale) {
+    const uint64_t count = (uint64_t)T * H * hd;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x) {
+        const int e = (int)(i % hd), head = (int)((i / hd) % H), pos = (int)(i / ((uint64_t)hd * H));
+        const size_t dst = (((size_t)page_table[pos / ps] * H + head) * ps + pos % ps) * hd + e;
+        cache[dst] = float_to_wt<WT>(gen_value(base, i, scale));
+    }
+}
+__global__ void fill_tokens_kernel(int* out, uint64_t base, int count, int vocab) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x)
+        out[i] = (int)(mix64(base + (uint64_t)i) % (uint64_t)vocab);
+}
+
+enum { TID_EMBED = 1, TID_HEAD = 2, TID_PROMPT = 3, TID_HIDDEN = 4, TID_GFINAL = 6, TID_DRAFT = 7, TID_LAYER_BASE = 100 };
+enum { K_WQKV = 0, K_WO = 1, K_WGATE = 2, K_WUP = 3, K_WDOWN = 4, K_G1 = 5, K_G2 = 6, K_KCACHE = 8, K_VCACHE = 9 };
+inline uint64_t layer_tid(int layer, int k) { return (uint64_t)TID_LAYER_BASE + 16ull * (uint64_t)layer + (uint64_t)k; }
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t off_layers, off_pt, off_kc, off_vc, off_h, off_feat, off_abuf, off_qkv, off_attn, off_act, off_po, off_ml,
+        off_cnt, off_hp, off_dbgd, off_dbgv, off_out, off_S, off_rlog, off_prompt, off_st, off_bar;
+    size_t off_embed, off_head, off_gfinal;
+    std::vector<size_t> off_w[5];     // wqkv, wo, wgate, wup, wdown
+    std::vector<size_t> off_g[2];
+    size_t total;
+};
+
+bool valid_config(const kg_config* c) {
+    if (!c || c->struct_size != sizeof(kg_config)) return false;
+    if (c->n_layers < 2 || c->exit_layer < 1 || c->exit_layer >= c->n_layers) return false;
+    if (c->d_model <= 0 || c->n_heads <= 0 || c->n_heads * c->head_dim != c->d_model) return false;
+    if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->d_model % 8 || c->d_ffn % 8 || c->d_ffn <= 0 || c->vocab <= 1) return false;
+    if (c->dtype != KG_F32 && c->dtype != KG_BF16) return false;
+    if (c->gamma_max < 1 || c->gamma_max > KG_GAMMA_MAX) return false;
+    if (c->page_size < 1 || c->max_seq < 2) return false;
+    if (c->n_heads > 256) return false;
+    // the plain path stages all rows of an operand in shared memory
+    const int kmax = c->d_ffn > c->d_model ? c->d_ffn : c->d_model;
+    const bool plain_everywhere = c->dtype == KG_F32 || (c->d_model % 32) || (c->d_ffn % 32);
+    if (plain_everywhere && (size_t)kmax * KG_M_MAX * 4 > (size_t)XS_BUDGET) return false;
+    return true;
+}
+
+Layout make_layout(const kg_config* c, int own_weights, int nctas) {
+    Layout L;
+    const size_t es = c->dtype == KG_BF16 ? 2 : 4;
+    const size_t d = c->d_model, F = c->d_ffn, V = c->vocab, H = c->n_heads, hd = c->head_dim;
+    const int nl = c->n_layers;
+    const size_t n_pages = (c->max_seq + c->page_size - 1) / c->page_size;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    L.off_st = take(sizeof(State));
+    L.off_bar = take(256);
+    L.off_layers = take(sizeof(LayerW) * (nl + 1));
+    L.off_pt = take(sizeof(int) * n_pages);
+    const size_t cache_bytes = (size_t)(nl + 1) * n_pages * H * c->page_size * hd * es;
+    L.off_kc = take(cache_bytes);
+    L.off_vc = take(cache_bytes);
+    L.off_h = take(4 * KG_M_MAX * d);
+    L.off_feat = take(4 * (KG_M_MAX + 1) * d);
+    L.off_abuf = take(4 * 2 * d);
+    L.off_qkv = take(4 * KG_M_MAX * 3 * d);
+    L.off_attn = take(4 * KG_M_MAX * d);
+    L.off_act = take(4 * KG_M_MAX * F);
+    L.off_po = take(4 * (size_t)KG_M_MAX * H * S_CAP * hd);
+    L.off_ml = take(4 * (size_t)KG_M_MAX * H * S_CAP * 2);
+    L.off_cnt = take(4 * H);
+    L.off_hp = take(sizeof(float4) * (size_t)nctas * KG_M_MAX);
+    L.off_dbgd = take(c->debug_logits ? 4 * (size_t)KG_M_MAX * V : 0);
+    L.off_dbgv = take(c->debug_logits ? 4 * (size_t)KG_M_MAX * V : 0);
+    L.off_out = take(4 * (size_t)(c->max_seq + KG_M_MAX));
+    L.off_S = take(4 * (size_t)(c->max_seq + KG_M_MAX));
+    L.off_rlog = take(16 * (size_t)(c->max_seq + KG_M_MAX));
+    L.off_prompt = take(4 * (size_t)c->max_seq);
+    for (int k = 0; k < 5; ++k) L.off_w[k].assign(nl + 1, 0);
+    for (int k = 0; k < 2; ++k) L.off_g[k].assign(nl + 1, 0);
+    L.off_embed = L.off_head = L.off_gfinal = 0;
+    if (own_weights) {
+        L.off_embed = take(es * V * d);
+        L.off_head = take(es * V * d);
+        L.off_gfinal = take(4 * d);
+        for (int i = 0; i <= nl; ++i) {
+            L.off_w[K_WQKV][i] = take(es * 3 * d * d);
+            L.off_w[K_WO][i] = take(es * d * d);
+            if (i < nl) {
+                L.off_w[K_WGATE][i] = take(es * F * d);
+                L.off_w[K_WUP][i] = take(es * F * d);
+                L.off_w[K_WDOWN][i] = take(es * d * F);
+            }
+            L.off_g[0][i] = take(4 * d);
+            L.off_g[1][i] = take(4 * d);
+        }
+    }
+    L.total = o;
+    return L;
+}
+
+int g_sm_count = 0;
+int sm_count() {
+    if (g_sm_count > 0) return g_sm_count;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    g_sm_count = n;
+    return n;
+}
+
+}  // namespace
+
+struct kg_model {
+    kg_config cfg;
+    Dev dev;
+    Layout lay;
+    char* arena;
+    cudaStream_t stream;
+    int nctas;
+    size_t smem;
+    bool own_weights;
+    bool prefilled, pending, ar_used, dead;
+    int gamma_pending;
+    long long P_upper;      // upper bound of the device-side position P
+    int force_simple;
+    std::vector<LayerW> layers_host;
+};
+
+#define CK(x) do { if ((x) != cudaSuccess) return KG_E_CUDA; } while (0)
+
+extern "C" const char* kg_strerror(int s) {
+    switch (s) {
+        case KG_OK: return "ok";
+        case KG_E_ARG: return "invalid argument";
+        case KG_E_STATE: return "call order violated";
+        case KG_E_NOMEM: return "arena too small";
+        case KG_E_SEQ_FULL: return "sequence would exceed max_seq";
+        case KG_E_CUDA: return "CUDA runtime error";
+        case KG_E_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" size_t kg_workspace_bytes(const kg_config* cfg, int own_weights) {
+    if (!valid_config(cfg)) return 0;
+    return make_layout(cfg, own_weights, sm_count()).total + 256;
+}
+
+template <typename WT>
+static int launch_program(kg_model* m, const Program& pg) {
+    CK(cudaMemsetAsync(m->dev.bar, 0, sizeof(unsigned), m->stream));
+    Program p = pg;
+    p.force_simple = m->force_simple;
+    void* args[] = {(void*)&m->dev, (void*)&p};
+    CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(NTHREADS), args, m->smem, m->stream));
+    return KG_OK;
+}
+static int launch(kg_model* m, const Program& pg) {
+    return m->cfg.dtype == KG_BF16 ? launch_program<__nv_bfloat16>(m, pg) : launch_program<float>(m, pg);
+}
+
+static int read_state(kg_model* m, State* out) {
+    CK(cudaMemcpyAsync(out, m->dev.st, sizeof(State), cudaMemcpyDeviceToHost, m->stream));
+    CK(cudaStreamSynchronize(m->stream));
+    if (out->status != 0) { m->dead = true; return out->status; }
+    return KG_OK;
+}
+
+template <typename WT>
+static int fill_weights(kg_model* m) {
+    const kg_config& c = m->cfg;
+    cudaStream_t s = m->stream;
+    const uint64_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+    const int nl = c.n_layers;
+    auto fill = [&](size_t off, uint64_t tid, uint64_t count, double std_) {
+        fill_matrix_kernel<WT><<<1184, 256, 0, s>>>(reinterpret_cast<WT*>(m->arena + off), stream_base(c.seed, tid), count, gen_scale(std_));
+    };
+    auto gain = [&](size_t off, uint64_t tid) {
+        fill_gain_kernel<<<16, 256, 0, s>>>(reinterpret_cast<float*>(m->arena + off), stream_base(c.seed, tid), (int)d, gen_scale(c.gain_std));
+    };
+    fill(m->lay.off_embed, TID_EMBED, V * d, c.embed_std);
+    fill(m->lay.off_head, TID_HEAD, V * d, c.init_std);
+    gain(m->lay.off_gfinal, TID_GFINAL);
+    for (int i = 0; i <= nl; ++i) {
+        const bool adapter = i == nl;
+        const double os = adapter ? c.adapter_resid_scale : (i >= c.exit_layer ? c.deep_resid_scale : 1.0);
+        // the output-projection std is formed in fp32 exactly as the host recipe does: float(init_std) * float(scale)
+        const double std_o = (double)c.init_std * os;
+        fill(m->lay.off_w[K_WQKV][i], layer_tid(i, K_WQKV), 3 * d * d, c.init_std);
+        fill(m->lay.off_w[K_WO][i], layer_tid(i, K_WO), d * d, std_o);
+        if (!adapter) {
+            fill(m->lay.off_w[K_WGATE][i], layer_tid(i, K_WGATE), F * d, c.init_std);
+            fill(m->lay.off_w[K_WUP][i], layer_tid(i, K_WUP), F * d, c.init_std);
+            fill(m->lay.off_w[K_WDOWN][i], layer_tid(i, K_WDOWN), d * F, std_o);
+        }
+        gain(m->lay.off_g[0][i], layer_tid(i, K_G1));
+        gain(m->lay.off_g[1][i], layer_tid(i, K_G2));
+    }
+    CK(cudaGetLastError());
+    return KG_OK;
+}
+
+extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* arena_dev, size_t arena_bytes,
+                             void* cuda_stream, kg_model** out) {
+    if (!out) return KG_E_ARG;
+    *out = nullptr;
+    if (!valid_config(cfg) || !arena_dev) return KG_E_ARG;
+    if (w) {
+        if (!w->embed_dev || !w->head_dev || !w->g_final_dev || !w->wqkv_dev || !w->wo_dev || !w->wgate_dev ||
+            !w->wup_dev || !w->wdown_dev || !w->g1_dev || !w->g2_dev) return KG_E_ARG;
+    }
+    const int nctas = sm_count();
+    const int own = w ? 0 : 1;
+    Layout lay = make_layout(cfg, own, nctas);
+    char* base = reinterpret_cast<char*>(align_up(reinterpret_cast<size_t>(arena_dev), 256));
+    if ((size_t)(base - reinterpret_cast<char*>(arena_dev)) + lay.total > arena_bytes) return KG_E_NOMEM;
+
+    kg_model* m = new (std::nothrow) kg_model();
+    if (!m) return KG_E_NOMEM;
+    m->cfg = *cfg; m->lay = lay; m->arena = base; m->stream = (cudaStream_t)cuda_stream; m->nctas = nctas;
+    m->own_weights = own != 0; m->prefilled = m->pending = m->ar_used = m->dead = false;
+    m->gamma_pending = 0; m->P_upper = 0; m->force_simple = 0;
+    m->smem = smem_bytes_needed();
+
+    const bool bf = cfg->dtype == KG_BF16;
+    const void* kfn = bf ? (const void*)kg_persistent_kernel<__nv_bfloat16> : (const void*)kg_persistent_kernel<float>;
+    if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m->smem) != cudaSuccess) { delete m; return KG_E_CUDA; }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kfn, NTHREADS, m->smem) != cudaSuccess || occ < 1) { delete m; return KG_E_CUDA; }
+
+    Dev& D = m->dev;
+    std::memset(&D, 0, sizeof(D));
+    D.dm.L = cfg->n_layers; D.dm.d = cfg->d_model; D.dm.H = cfg->n_heads; D.dm.hd = cfg->head_dim; D.dm.F = cfg->d_ffn;
+    D.dm.V = cfg->vocab; D.dm.l = cfg->exit_layer; D.dm.eps = cfg->rms_eps; D.dm.theta = cfg->rope_theta;
+    D.dm.logit_scale = cfg->logit_scale; D.dm.max_seq = cfg->max_seq; D.dm.page_size = cfg->page_size;
+    D.dm.n_pages = (cfg->max_seq + cfg->page_size - 1) / cfg->page_size; D.dm.gamma_max = cfg->gamma_max;
+    D.dm.debug = cfg->debug_logits;
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        D.inv_freq[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
+    auto P = [&](size_t off) { return base + off; };
+    D.st = (State*)P(lay.off_st); D.bar = (unsigned*)P(lay.off_bar);
+    D.layers = (const LayerW*)P(lay.off_layers); D.page_table = (const int*)P(lay.off_pt);
+    D.kcache = P(lay.off_kc); D.vcache = P(lay.off_vc);
+    D.h = (float*)P(lay.off_h); D.feat = (float*)P(lay.off_feat); D.abuf = (float*)P(lay.off_abuf);
+    D.qkv = (float*)P(lay.off_qkv); D.attn = (float*)P(lay.off_attn); D.act = (float*)P(lay.off_act);
+    D.att_po = (float*)P(lay.off_po); D.att_ml = (float*)P(lay.off_ml); D.att_cnt = (unsigned*)P(lay.off_cnt);
+    D.head_part = (float4*)P(lay.off_hp);
+    D.dbg_draft = cfg->debug_logits ? (float*)P(lay.off_dbgd) : nullptr;
+    D.dbg_verify = cfg->debug_logits ? (float*)P(lay.off_dbgv) : nullptr;
+    D.out_tokens = (int*)P(lay.off_out); D.S = (int*)P(lay.off_S); D.round_log = (int*)P(lay.off_rlog);
+    D.prompt = (const int*)P(lay.off_prompt);
+
+    const int nl = cfg->n_layers;
+    m->layers_host.resize(nl + 1);
+    if (own) {
+        D.embed = P(lay.off_embed); D.head = P(lay.off_head); D.g_final = (const float*)P(lay.off_gfinal);
+        for (int i = 0; i <= nl; ++i) {
+            LayerW& lw = m->layers_host[i];
+            lw.wqkv = P(lay.off_w[K_WQKV][i]); lw.wo = P(lay.off_w[K_WO][i]);
+            lw.wgate = i < nl ? P(lay.off_w[K_WGATE][i]) : nullptr;
+            lw.wup = i < nl ? P(lay.off_w[K_WUP][i]) : nullptr;
+            lw.wdown = i < nl ? P(lay.off_w[K_WDOWN][i]) : nullptr;
+            lw.g1 = (const float*)P(lay.off_g[0][i]); lw.g2 = (const float*)P(lay.off_g[1][i]);
+        }
+    } else {
+        D.embed = w->embed_dev; D.head = w->head_dev; D.g_final = w->g_final_dev;
+        for (int i = 0; i <= nl; ++i) {
+            LayerW& lw = m->layers_host[i];
+            lw.wqkv = w->wqkv_dev[i]; lw.wo = w->wo_dev[i];
+            lw.wgate = i < nl ? w->wgate_dev[i] : nullptr;
+            lw.wup = i < nl ? w->wup_dev[i] : nullptr;
+            lw.wdown = i < nl ? w->wdown_dev[i] : nullptr;
+            lw.g1 = w->g1_dev[i]; lw.g2 = w->g2_dev[i];
+            if (!lw.wqkv || !lw.wo || !lw.g1 || !lw.g2 || (i < nl && (!lw.wgate || !lw.wup || !lw.wdown))) { delete m; return KG_E_ARG; }
+        }
+    }
+    cudaStream_t s = m->stream;
+    bool ok = cudaMemcpyAsync(P(lay.off_layers), m->layers_host.data(), sizeof(LayerW) * (nl + 1), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    // page table: identity, or a fixed permutation (reversal within blocks of 4 pages plus a rotation)
+    std::vector<int> pt(D.dm.n_pages);
+    for (int i = 0; i < D.dm.n_pages; ++i) pt[i] = i;
+    if (cfg->page_shuffle) {
+        const int n = D.dm.n_pages;
+        for (int i = 0; i < n; ++i) pt[i] = (int)(((long long)i * 7 + 3) % n);
+        // i -> 7i+3 mod n is a permutation only if gcd(7, n) == 1; otherwise fall back to reversal
+        if (n % 7 == 0) for (int i = 0; i < n; ++i) pt[i] = n - 1 - i;
+    }
+    ok = ok && cudaMemcpyAsync(P(lay.off_pt), pt.data(), sizeof(int) * pt.size(), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(D.st, 0, sizeof(State), s) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(D.att_cnt, 0, 4 * cfg->n_heads, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;    // pt / layers_host are host temporaries
+    if (!ok) { delete m; return KG_E_CUDA; }
+    if (own) {
+        int r = bf ? fill_weights<__nv_bfloat16>(m) : fill_weights<float>(m);
+        if (r != KG_OK) { delete m; return r; }
+    }
+    *out = m;
+    return KG_OK;
+}
+
+extern "C" int kg_free_model(kg_model* m) {
+    if (!m) return KG_E_ARG;
+    delete m;
+    return KG_OK;
+}
+
+extern "C" int kg_reset(kg_model* m) {
+    if (!m) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    CK(cudaMemsetAsync(m->dev.st, 0, sizeof(State), m->stream));
+    CK(cudaMemsetAsync(m->dev.att_cnt, 0, 4 * m->cfg.n_heads, m->stream));
+    m->prefilled = m->pending = m->ar_used = false;
+    m->P_upper = 0;
+    return KG_OK;
+}
+
+static int prefill_common(kg_model* m, int32_t n) {
+    Program pg{}; pg.kind = PROG_PREFILL; pg.n = n;
+    int r = launch(m, pg);
+    if (r != KG_OK) return r;
+    m->prefilled = true; m->pending = false; m->P_upper = n;
+    return KG_OK;
+}
+
+extern "C" int kg_prefill(kg_model* m, const int32_t* prompt_host, int32_t n, int32_t* first_token_host) {
+    if (!m || !prompt_host || n < 1) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (m->prefilled || m->ar_used) return KG_E_STATE;
+    if (n + 1 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    for (int i = 0; i < n; ++i) if (prompt_host[i] < 0 || prompt_host[i] >= m->cfg.vocab) return KG_E_ARG;
+    CK(cudaMemcpyAsync((void*)m->dev.prompt, prompt_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, m->stream));
+    int r = prefill_common(m, n);
+    if (r != KG_OK) return r;
+    if (first_token_host) {
+        State st;
+        r = read_state(m, &st);
+        if (r != KG_OK) return r;
+        *first_token_host = st.x0;
+    } else {
+        // the prompt buffer is the caller's: make sure the copy has left it
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_prefill_device(kg_model* m, const int32_t* prompt_dev, int32_t n) {
+    if (!m || !prompt_dev || n < 1) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (m->prefilled || m->ar_used) return KG_E_STATE;
+    if (n + 1 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    CK(cudaMemcpyAsync((void*)m->dev.prompt, prompt_dev, sizeof(int32_t) * n, cudaMemcpyDeviceToDevice, m->stream));
+    return prefill_common(m, n);
+}
+
+static bool bad_spec(const kg_model* m, float eta, int gamma, int mode) {
+    return !(eta == eta) || gamma < 1 || gamma > m->cfg.gamma_max || (mode != KG_STOP_KEEP && mode != KG_STOP_DROP);
+}
+
+extern "C" int kg_draft(kg_model* m, float eta, int32_t gamma, int32_t stop_mode, kg_draft_out* out) {
+    if (!m || bad_spec(m, eta, gamma, stop_mode)) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (!m->prefilled || m->pending || m->ar_used) return KG_E_STATE;
+    if (m->P_upper + gamma + 2 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    Program pg{}; pg.kind = PROG_DRAFT; pg.eta = eta; pg.gamma = gamma; pg.stop_mode = stop_mode;
+    int r = launch(m, pg);
+    if (r != KG_OK) return r;
+    m->pending = true; m->gamma_pending = gamma;
+    if (out) {
+        State st;
+        r = read_state(m, &st);
+        if (r != KG_OK) return r;
+        out->n_drafted = st.n_d; out->n_steps = st.n_steps;
+        for (int i = 0; i < KG_GAMMA_MAX; ++i) { out->tokens[i] = i < st.n_d ? st.draft_tok[i] : -1; out->conf[i] = i < st.n_steps ? st.conf[i] : 0.f; }
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_verify(kg_model* m, kg_verify_out* out) {
+    if (!m) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (!m->prefilled || !m->pending) return KG_E_STATE;
+    Program pg{}; pg.kind = PROG_VERIFY;
+    int r = launch(m, pg);
+    if (r != KG_OK) return r;
+    m->pending = false;
+    m->P_upper += m->gamma_pending + 1;
+    if (out) {
+        State st;
+        r = read_state(m, &st);
+        if (r != KG_OK) return r;
+        out->n_rows = st.M; out->n_accept = st.k_acc; out->n_emitted = st.n_emit;
+        for (int i = 0; i < KG_M_MAX; ++i) { out->emitted[i] = i < st.n_emit ? st.emitted[i] : -1; out->target[i] = i < st.M ? st.target[i] : -1; }
+        m->P_upper = st.P;
+    }
+    return KG_OK;
+}
+
+static void fill_stats(kg_model* m, const State& st, const std::vector<int>& S, int max_tokens, kg_stats* out) {
+    std::memset(out, 0, sizeof(*out));
+    std::vector<int> s2(S);
+    // truncate so that only tokens up to max_tokens (x_0 excluded from S) are counted
+    long long sum = 0;
+    for (size_t i = 0; i < s2.size(); ++i) {
+        if (max_tokens >= 0 && sum + s2[i] > max_tokens - 1) { s2[i] = (int)(max_tokens - 1 - sum); s2.resize(s2[i] > 0 ? i + 1 : i); sum = max_tokens - 1; break; }
+        sum += s2[i];
+    }
+    out->rounds = (int)s2.size(); out->tokens = (int)sum;
+    out->draft_steps = st.draft_steps_total; out->drafted = st.drafted_total; out->accepted = st.accepted_total;
+    if (!s2.empty()) {
+        out->cr = (double)sum / (double)s2.size();
+        for (int w = 0; w <= KG_M_MAX; ++w) {
+            int cnt = 0;
+            for (int v : s2) cnt += (v - w > 0);
+            out->ctar[w] = (double)cnt / (double)s2.size();
+        }
+    }
+}
+
+static int read_S_vec(kg_model* m, int rounds, std::vector<int>& S) {
+    S.assign(rounds, 0);
+    if (rounds > 0) {
+        CK(cudaMemcpyAsync(S.data(), m->dev.S, sizeof(int) * rounds, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_decode(kg_model* m, int32_t max_new, float eta, int32_t gamma, int32_t stop_mode, kg_stats* stats) {
+    if (!m || bad_spec(m, eta, gamma, stop_mode) || max_new < 1) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (!m->prefilled || m->pending || m->ar_used) return KG_E_STATE;
+    if (m->P_upper + max_new + gamma + 2 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    Program pg{}; pg.kind = PROG_DECODE; pg.n = max_new; pg.eta = eta; pg.gamma = gamma; pg.stop_mode = stop_mode;
+    int r = launch(m, pg);
+    if (r != KG_OK) return r;
+    m->P_upper += max_new + gamma + 1;
+    if (stats) {
+        State st;
+        r = read_state(m, &st);
+        if (r != KG_OK) return r;
+        m->P_upper = st.P;
+        std::vector<int> S;
+        r = read_S_vec(m, st.rounds, S);
+        if (r != KG_OK) return r;
+        fill_stats(m, st, S, max_new, stats);
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_decode_ar(kg_model* m, int32_t n_tokens, int32_t* out_host) {
+    if (!m || n_tokens < 1) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    if (!m->prefilled || m->pending) return KG_E_STATE;
+    if (m->P_upper + n_tokens + 1 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    Program pg{}; pg.kind = PROG_AR; pg.n = n_tokens;
+    int r = launch(m, pg);
+    if (r != KG_OK) return r;
+    m->ar_used = true;
+    m->P_upper += n_tokens;
+    if (out_host) {
+        State st;
+        r = read_state(m, &st);
+        if (r != KG_OK) return r;
+        CK(cudaMemcpyAsync(out_host, m->dev.out_tokens, sizeof(int) * n_tokens, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_read_tokens(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out) {
+    if (!m || !out_host || max_n < 0) return KG_E_ARG;
+    State st;
+    int r = read_state(m, &st);
+    if (r != KG_OK) return r;
+    const int n = st.total < max_n ? st.total : max_n;
+    if (n > 0) {
+        CK(cudaMemcpyAsync(out_host, m->dev.out_tokens, sizeof(int) * n, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    if (n_out) *n_out = n;
+    return KG_OK;
+}
+
+extern "C" int kg_read_S(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out) {
+    if (!m || !out_host || max_n < 0) return KG_E_ARG;
+    State st;
+    int r = read_state(m, &st);
+    if (r != KG_OK) return r;
+    const int n = st.rounds < max_n ? st.rounds : max_n;
+    if (n > 0) {
+        CK(cudaMemcpyAsync(out_host, m->dev.S, sizeof(int) * n, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    if (n_out) *n_out = n;
+    return KG_OK;
+}
+
+extern "C" int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_prompt, int32_t max_new,
+                           float eta, int32_t gamma, int32_t stop_mode,
+                           int32_t* out_tokens_host, int32_t* n_out, kg_stats* stats) {
+    if (!m || !prompt_host || !out_tokens_host || max_new < 1 || bad_spec(m, eta, gamma, stop_mode)) return KG_E_ARG;
+    if ((long long)n_prompt + max_new + gamma + 2 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    int r = kg_reset(m);
+    if (r != KG_OK) return r;
+    for (int i = 0; i < n_prompt; ++i) if (prompt_host[i] < 0 || prompt_host[i] >= m->cfg.vocab) return KG_E_ARG;
+    if (n_prompt < 1) return KG_E_ARG;
+    CK(cudaMemcpyAsync((void*)m->dev.prompt, prompt_host, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->stream));
+    r = prefill_common(m, n_prompt);
+    if (r != KG_OK) return r;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    const bool timed = stats != nullptr;
+    if (timed) { CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1)); CK(cudaEventRecord(e0, m->stream)); }
+    r = kg_decode(m, max_new, eta, gamma, stop_mode, nullptr);
+    if (timed && r == KG_OK) cudaEventRecord(e1, m->stream);
+    State st;
+    if (r == KG_OK) r = read_state(m, &st);
+    if (r == KG_OK) {
+        if (cudaMemcpyAsync(out_tokens_host, m->dev.out_tokens, sizeof(int) * max_new, cudaMemcpyDeviceToHost, m->stream) != cudaSuccess ||
+            cudaStreamSynchronize(m->stream) != cudaSuccess) r = KG_E_CUDA;
+    }
+    if (r == KG_OK) {
+        m->P_upper = st.P;
+        if (n_out) *n_out = max_new;
+        if (stats) {
+            std::vector<int> S;
+            r = read_S_vec(m, st.rounds, S);
+            if (r == KG_OK) {
+                fill_stats(m, st, S, max_new, stats);
+                float ms = 0.f;
+                if (cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess) stats->ms_decode = ms;
+            }
+        }
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    return r;
+}
+
+extern "C" int kg_debug_logits(kg_model* m, int32_t which, int32_t row, float* out_host) {
+    if (!m || !out_host || row < 0 || row >= KG_M_MAX || (which != 0 && which != 1)) return KG_E_ARG;
+    if (!m->cfg.debug_logits) return KG_E_STATE;
+    const float* src = (which == 0 ? m->dev.dbg_draft : m->dev.dbg_verify) + (size_t)row * m->cfg.vocab;
+    CK(cudaMemcpyAsync(out_host, src, sizeof(float) * m->cfg.vocab, cudaMemcpyDeviceToHost, m->stream));
+    CK(cudaStreamSynchronize(m->stream));
+    return KG_OK;
+}
+
+extern "C" int kg_read_weight(kg_model* m, const char* name, int32_t layer, uint64_t offset, uint64_t count, float* out_host) {
+    if (!m || !name || !out_host) return KG_E_ARG;
+    const kg_config& c = m->cfg;
+    const uint64_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+    const void* p = nullptr; uint64_t n = 0; bool f32 = false;
+    const bool lay_ok = layer >= 0 && layer <= c.n_layers;
+    if (!std::strcmp(name, "embed")) { p = m->dev.embed; n = V * d; }
+    else if (!std::strcmp(name, "head")) { p = m->dev.head; n = V * d; }
+    else if (!std::strcmp(name, "g_final")) { p = m->dev.g_final; n = d; f32 = true; }
+    else if (!lay_ok) return KG_E_ARG;
+    else if (!std::strcmp(name, "wqkv")) { p = m->layers_host[layer].wqkv; n = 3 * d * d; }
+    else if (!std::strcmp(name, "wo")) { p = m->layers_host[layer].wo; n = d * d; }
+    else if (!std::strcmp(name, "wgate")) { p = m->layers_host[layer].wgate; n = F * d; }
+    else if (!std::strcmp(name, "wup")) { p = m->layers_host[layer].wup; n = F * d; }
+    else if (!std::strcmp(name, "wdown")) { p = m->layers_host[layer].wdown; n = d * F; }
+    else if (!std::strcmp(name, "g1")) { p = m->layers_host[layer].g1; n = d; f32 = true; }
+    else if (!std::strcmp(name, "g2")) { p = m->layers_host[layer].g2; n = d; f32 = true; }
+    else return KG_E_ARG;
+    if (!p || offset > n || count > n - offset) return KG_E_ARG;
+    if (f32 || c.dtype == KG_F32) {
+        CK(cudaMemcpyAsync(out_host, (const float*)p + offset, 4 * count, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    } else {
+        std::vector<uint16_t> tmp(count);
+        CK(cudaMemcpyAsync(tmp.data(), (const uint16_t*)p + offset, 2 * count, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+        for (uint64_t i = 0; i < count; ++i) { uint32_t b = (uint32_t)tmp[i] << 16; std::memcpy(out_host + i, &b, 4); }
+    }
+    return KG_OK;
+}
+
+extern "C" int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t seed) {
+    if (!m || T < 1 || n_d < -1 || n_d > m->cfg.gamma_max) return KG_E_ARG;
+    if (m->dead) return KG_E_TIMEOUT;
+    const kg_config& c = m->cfg;
+    if (T + c.gamma_max + 2 > c.max_seq) return KG_E_SEQ_FULL;
+    cudaStream_t s = m->stream;
+    const float one = gen_scale(1.0);
+    const size_t lstride = (size_t)m->dev.dm.n_pages * c.n_heads * c.page_size * c.head_dim;
+    for (int i = 0; i <= c.n_layers; ++i) {
+        if (c.dtype == KG_BF16) {
+            fill_cache_kernel<__nv_bfloat16><<<592, 256, 0, s>>>((__nv_bfloat16*)m->dev.kcache + i * lstride, m->dev.page_table, stream_base(seed, layer_tid(i, K_KCACHE)), T, c.n_heads, c.head_dim, c.page_size, one);
+            fill_cache_kernel<__nv_bfloat16><<<592, 256, 0, s>>>((__nv_bfloat16*)m->dev.vcache + i * lstride, m->dev.page_table, stream_base(seed, layer_tid(i, K_VCACHE)), T, c.n_heads, c.head_dim, c.page_size, one);
+        } else {
+            fill_cache_kernel<float><<<592, 256, 0, s>>>((float*)m->dev.kcache + i * lstride, m->dev.page_table, stream_base(seed, layer_tid(i, K_KCACHE)), T, c.n_heads, c.head_dim, c.page_size, one);
+            fill_cache_kernel<float><<<592, 256, 0, s>>>((float*)m->dev.vcache + i * lstride, m->dev.page_table, stream_base(seed, layer_tid(i, K_VCACHE)), T, c.n_heads, c.head_dim, c.page_size, one);
+        }
+    }
+    fill_f32_kernel<<<64, 256, 0, s>>>(m->dev.feat, stream_base(seed, TID_HIDDEN), (uint64_t)(KG_M_MAX + 1) * c.d_model, one);
+    CK(cudaGetLastError());
+    // tokens: x_0 and the drafts
+    const uint64_t tb = stream_base(seed, TID_DRAFT);
+    State st;
+    std::memset(&st, 0, sizeof(st));
+    st.P = T; st.len_A = T; st.total = 1; st.x0 = (int)(mix64(tb + 1000) % (uint64_t)c.vocab);
+    if (n_d >= 0) {
+        st.pending = 1; st.n_d = n_d; st.n_steps = n_d;
+        for (int i = 0; i < n_d; ++i) { st.draft_tok[i] = (int)(mix64(tb + (uint64_t)i) % (uint64_t)c.vocab); st.conf[i] = 1.0f; }
+    }
+    CK(cudaMemcpyAsync(m->dev.st, &st, sizeof(State), cudaMemcpyHostToDevice, s));
+    CK(cudaMemsetAsync(m->dev.att_cnt, 0, 4 * c.n_heads, s));
+    CK(cudaStreamSynchronize(s));
+    m->prefilled = true; m->pending = n_d >= 0; m->ar_used = false; m->gamma_pending = n_d >= 0 ? n_d : 0; m->P_upper = T;
+    return KG_OK;
+}
+
+// Test hook (not in the public header): route bf16 linears through the plain path.
+extern "C" int kg_debug_force_simple(kg_model* m, int on) {
+    if (!m) return KG_E_ARG;
+    m->force_simple = on ? 1 : 0;
+    return KG_OK;
+}
+
+// ------------------------------------------------------------------------------------ single operators
+namespace {
+
+struct OpScratch { size_t off_hp, off_po, off_ml, off_cnt, off_pt, total; };
+OpScratch op_layout() {
+    OpScratch s; size_t o = 0;
+    auto take = [&](size_t b) { size_t r = o; o = align_up(o + b, 256); return r; };
+    s.off_hp = take(sizeof(float4) * 1024 * KG_M_MAX);
+    s.off_po = take(4 * (size_t)KG_M_MAX * S_CAP * 8192);
+    s.off_ml = take(4 * (size_t)KG_M_MAX * 256 * S_CAP * 2);
+    s.off_cnt = take(4 * 256);
+    s.total = o;
+    return s;
+}
+
+template <typename WT>
+__global__ void __launch_bounds__(NTHREADS, 1) op_linear_kernel(LinArgs a, State* st, int force_simple) {
+    extern __shared__ __align__(128) char smem[];
+    Ctx c; c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = nullptr; c.smem = smem; c.grid = false;
+    LinDispatch<WT>::run(a, c, force_simple != 0);
+}
+__global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* tok, float* p) {
+    if (threadIdx.x < M) { int t; float pp; head_final(part, nctas, threadIdx.x, t, pp); tok[threadIdx.x] = t; p[threadIdx.x] = pp; }
+}
+template <typename WT>
+__global__ void __launch_bounds__(NTHREADS, 1) op_attention_kernel(const __grid_constant__ Dev D, AttArgs a) {
+    extern __shared__ __align__(128) char smem[];
+    Ctx c; c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = nullptr; c.bar = nullptr; c.smem = smem; c.grid = false;
+    attention_op<WT>(D, a, c);
+}
+
+int g_force_simple_ops = 0;
+
+template <typename K>
+int set_smem(K kfn) {
+    return cudaFuncSetAttribute((const void*)kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_needed()) == cudaSuccess ? KG_OK : KG_E_CUDA;
+}
+
+}  // namespace
+
+extern "C" size_t kg_op_scratch_bytes(void) { return op_layout().total; }
+
+extern "C" int kg_debug_force_simple_ops(int on) { g_force_simple_ops = on ? 1 : 0; return KG_OK; }
+
+static int op_linear_common(int32_t dtype, LinArgs& a, cudaStream_t s) {
+    if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
+    if (a.M < 1 || a.M > KG_M_MAX || a.N < 1 || a.K < 8 || (a.K % 8)) return KG_E_ARG;
+    const bool plain = dtype == KG_F32 || g_force_simple_ops || (a.K % 32);
+    if (plain && (size_t)a.K * a.M * 4 > (size_t)XS_BUDGET) return KG_E_ARG;
+    const int nctas = sm_count();
+    if (dtype == KG_BF16) {
+        if (set_smem(op_linear_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
+        op_linear_kernel<__nv_bfloat16><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(a, nullptr, g_force_simple_ops);
+    } else {
+        if (set_smem(op_linear_kernel<float>) != KG_OK) return KG_E_CUDA;
+        op_linear_kernel<float><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(a, nullptr, g_force_simple_ops);
+    }
+    CK(cudaGetLastError());
+    return KG_OK;
+}
+
+extern "C" int kg_op_linear(int32_t dtype, const void* W, const void* W2, int32_t N, int32_t K,
+                            const float* x, int32_t M, const float* gain, float eps,
+                            const float* resid, int32_t swiglu, float* out, void* scratch, void* stream) {
+    if (!W || !x || !out || !scratch) return KG_E_ARG;
+    if (swiglu && !W2) return KG_E_ARG;
+    LinArgs a{};
+    a.W = W; a.W2 = swiglu ? W2 : nullptr; a.N = N; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
+    a.resid = resid; a.ldr = N; a.out = out; a.ldo = N;
+    a.epi = swiglu ? EPI_SWIGLU : (resid ? EPI_RESID : EPI_STORE);
+    return op_linear_common(dtype, a, (cudaStream_t)stream);
+}
+
+extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K, const float* x, int32_t M,
+                             const float* gain, float eps, float logit_scale,
+                             int32_t* tok, float* p, float* logits, void* scratch, void* stream) {
+    if (!W || !x || !tok || !p || !scratch) return KG_E_ARG;
+    if (sm_count() > 1024) return KG_E_ARG;
+    OpScratch sc = op_layout();
+    LinArgs a{};
+    a.W = W; a.N = V; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
+    a.epi = EPI_HEAD; a.scale = logit_scale; a.head_part = (float4*)((char*)scratch + sc.off_hp);
+    a.logits_dbg = logits; a.ld_dbg = V;
+    int r = op_linear_common(dtype, a, (cudaStream_t)stream);
+    if (r != KG_OK) return r;
+    op_head_final_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(a.head_part, sm_count(), M, tok, p);
+    CK(cudaGetLastError());
+    return KG_OK;
+}
+
+extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32_t pos0, int32_t H, int32_t hd,
+                               float theta, void* kc, void* vc, const int32_t* page_table, int32_t page_size,
+                               float* out, void* scratch, void* stream) {
+    if (!qkv || !kc || !vc || !page_table || !out || !scratch) return KG_E_ARG;
+    if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
+    if (M < 1 || M > KG_M_MAX || pos0 < 0 || H < 1 || H > 256 || (hd != 32 && hd != 64 && hd != 128) || page_size < 1) return KG_E_ARG;
+    if ((size_t)H * hd > 8192) return KG_E_ARG;
+    OpScratch sc = op_layout();
+    cudaStream_t s = (cudaStream_t)stream;
+    Dev D;
+    std::memset(&D, 0, sizeof(D));
+    D.dm.H = H; D.dm.hd = hd; D.dm.d = H * hd; D.dm.page_size = page_size; D.dm.theta = theta;
+    for (int i = 0; i < hd / 2; ++i) D.inv_freq[i] = std::pow((double)theta, -2.0 * (double)i / (double)hd);
+    D.page_table = page_table;
+    D.att_po = (float*)((char*)scratch + sc.off_po); D.att_ml = (float*)((char*)scratch + sc.off_ml);
+    D.att_cnt = (unsigned*)((char*)scratch + sc.off_cnt);
+    CK(cudaMemsetAsync(D.att_cnt, 0, 4 * 256, s));
+    AttArgs a; a.qkv = qkv; a.M = M; a.pos0 = pos0; a.kc = kc; a.vc = vc; a.out = out;
+    const int nctas = sm_count();
+    if (dtype == KG_BF16) {
+        if (set_smem(op_attention_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
+        op_attention_kernel<__nv_bfloat16><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(D, a);
+    } else {
+        if (set_smem(op_attention_kernel<float>) != KG_OK) return KG_E_CUDA;
+        op_attention_kernel<float><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(D, a);
+    }
+    CK(cudaGetLastError());
+    return KG_OK;
+}

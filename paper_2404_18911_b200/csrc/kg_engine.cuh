@@ -1,0 +1,288 @@
+// The persistent decode kernel: one cooperative grid (one CTA per SM) runs whole phases of the
+// method - prefill chunks, the draft loop with its on-device exit test, the verify pass, the
+// prefix accept / rollback, or many rounds back to back - with grid barriers between dependent
+// operators and no host involvement.
+#pragma once
+
+#include "kg_device.cuh"
+
+namespace kg {
+
+enum { PROG_PREFILL = 0, PROG_DRAFT = 1, PROG_VERIFY = 2, PROG_DECODE = 3, PROG_AR = 4 };
+
+struct Program {
+    int kind;
+    int n;              // PREFILL: prompt length; DECODE / AR: total tokens wanted (x_0 included)
+    float eta; int gamma; int stop_mode;
+    int force_simple;   // 1: route bf16 linears through the plain path (cross-check)
+};
+
+#define KG_SYNC(where) do { if (!grid_sync(c, (where))) return false; } while (0)
+
+template <typename WT>
+struct Engine {
+    const Dev& D;
+    Ctx& c;
+    const Program& pg;
+
+    __device__ Engine(const Dev& d, Ctx& cx, const Program& p) : D(d), c(cx), pg(p) {}
+
+    __device__ __forceinline__ void linear(const LinArgs& a) { LinDispatch<WT>::run(a, c, pg.force_simple != 0); }
+
+    __device__ size_t cache_layer_stride() const {
+        return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
+    }
+
+    // h[i] = E[token_i]
+    __device__ void embed_rows(const int* toks_global, int tok_single, int M, float* out) {
+        const int d = D.dm.d;
+        const WT* E = reinterpret_cast<const WT*>(D.embed);
+        for (int idx = c.cta * NTHREADS + threadIdx.x; idx < M * d; idx += c.nctas * NTHREADS) {
+            const int i = idx / d, e = idx % d;
+            const int tok = toks_global ? __ldcg(toks_global + i) : tok_single;
+            out[idx] = wt_to_float<WT>(E[(size_t)tok * d + e]);
+        }
+    }
+
+    // One decoder block on M rows at positions pos0.. (Section 3.1's M^b layers):
+    //   h  = x + Wo Attn(RMSNorm(x; g1));   out = h + Wdown(SiLU(Wgate n) * Wup n), n = RMSNorm(h; g2)
+    __device__ bool run_layer(int li, int M, int pos0, const float* xin, float* out) {
+        const Dims& dm = D.dm;
+        const LayerW lw = D.layers[li];
+        LinArgs a{};
+        a.M = M; a.eps = dm.eps;
+        // q, k, v
+        a.W = lw.wqkv; a.W2 = nullptr; a.N = 3 * dm.d; a.K = dm.d;
+        a.x = xin; a.ldx = dm.d; a.gain = lw.g1; a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
+        linear(a);
+        KG_SYNC(10);
+        AttArgs at;
+        at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
+        at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)li * cache_layer_stride();
+        at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)li * cache_layer_stride();
+        at.out = D.attn;
+        attention_op<WT>(D, at, c);
+        KG_SYNC(11);
+        // output projection + residual -> h
+        a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
+        a.epi = EPI_RESID; a.resid = xin; a.ldr = dm.d; a.out = D.h; a.ldo = dm.d;
+        linear(a);
+        KG_SYNC(12);
+        // SwiGLU
+        a.W = lw.wgate; a.W2 = lw.wup; a.N = dm.F; a.K = dm.d; a.x = D.h; a.ldx = dm.d; a.gain = lw.g2;
+        a.epi = EPI_SWIGLU; a.out = D.act; a.ldo = dm.F;
+        linear(a);
+        KG_SYNC(13);
+        a.W = lw.wdown; a.W2 = nullptr; a.N = dm.d; a.K = dm.F; a.x = D.act; a.ldx = dm.F; a.gain = nullptr;
+        a.epi = EPI_RESID; a.resid = D.h; a.ldr = dm.d; a.out = out; a.ldo = dm.d;
+        linear(a);
+        KG_SYNC(14);
+        return true;
+    }
+
+    // Adapter A (Section 3.1, Table 2): a = f + W^A_o Attn(RMSNorm(f; g_in)) on rows f[M] at pos0..;
+    // with want_out == false only the adapter's K/V are appended (prefill).
+    __device__ bool run_adapter(int M, int pos0, const float* f, bool want_out) {
+        const Dims& dm = D.dm;
+        const LayerW lw = D.layers[dm.L];
+        LinArgs a{};
+        a.M = M; a.eps = dm.eps;
+        a.W = lw.wqkv; a.N = 3 * dm.d; a.K = dm.d; a.x = f; a.ldx = dm.d; a.gain = lw.g1;
+        a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
+        linear(a);
+        KG_SYNC(20);
+        AttArgs at;
+        at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
+        at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)dm.L * cache_layer_stride();
+        at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)dm.L * cache_layer_stride();
+        at.out = D.attn;
+        attention_op<WT>(D, at, c);
+        KG_SYNC(21);
+        if (!want_out) return true;
+        a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
+        a.epi = EPI_RESID; a.resid = f; a.ldr = dm.d; a.out = D.abuf; a.ldo = dm.d;
+        linear(a);
+        KG_SYNC(22);
+        return true;
+    }
+
+    // Shared LM head on rows x[M] (norm gain `gain`), then the merged (token, p) per row, the same
+    // values in every thread of every CTA.
+    __device__ bool run_head(const float* x, int M, const float* gain, float* dbg, int* toks, float* ps) {
+        const Dims& dm = D.dm;
+        LinArgs a{};
+        a.M = M; a.eps = dm.eps;
+        a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = x; a.ldx = dm.d; a.gain = gain;
+        a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
+        a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
+        linear(a);
+        KG_SYNC(30);
+        __shared__ int s_tok[M_MAX];
+        __shared__ float s_p[M_MAX];
+        if (threadIdx.x < M) {
+            int tk; float p;
+            head_final(D.head_part, c.nctas, threadIdx.x, tk, p);
+            s_tok[threadIdx.x] = tk; s_p[threadIdx.x] = p;
+        }
+        __syncthreads();
+        for (int i = 0; i < M; ++i) { toks[i] = s_tok[i]; ps[i] = s_p[i]; }
+        __syncthreads();
+        return true;
+    }
+
+    // ---- sequence state, replicated: every thread of every CTA holds the same values -----------
+    int P, len_A, x0, total, rounds;
+    int n_d, n_steps;
+    int dtok[M_MAX];
+    float dconf[M_MAX];
+
+    __device__ void load_state() {
+        P = __ldcg(&D.st->P); len_A = __ldcg(&D.st->len_A); x0 = __ldcg(&D.st->x0);
+        total = __ldcg(&D.st->total); rounds = __ldcg(&D.st->rounds);
+        n_d = __ldcg(&D.st->n_d); n_steps = __ldcg(&D.st->n_steps);
+        for (int i = 0; i < M_MAX; ++i) { dtok[i] = __ldcg(&D.st->draft_tok[i]); dconf[i] = __ldcg(&D.st->conf[i]); }
+    }
+    __device__ bool leader() const { return c.cta == 0 && threadIdx.x == 0; }
+
+    // early feature of token `tok` at position pos -> feat slot
+    __device__ bool shallow_pass(int tok, int pos, int slot) {
+        const Dims& dm = D.dm;
+        embed_rows(nullptr, tok, 1, D.h);
+        KG_SYNC(1);
+        for (int i = 0; i < dm.l; ++i)
+            if (!run_layer(i, 1, pos, D.h, (i == dm.l - 1) ? D.feat + (size_t)slot * dm.d : D.h)) return false;
+        return true;
+    }
+
+    // Draft phase of one round (Section 3.2; Eq. 4; Figure 2).
+    __device__ bool draft_phase() {
+        const Dims& dm = D.dm;
+        n_d = 0; n_steps = 0;
+        int cur = x0;
+        bool stop_after_shallow = false;
+        while (true) {
+            if (!shallow_pass(cur, P + n_d, 1 + n_d)) return false;                 // f[n_d]
+            if (n_d == pg.gamma || stop_after_shallow) break;
+            const int MA = P + n_d - len_A + 1;                                     // 1, or 2 when the adapter cache lags
+            const float* f = D.feat + (size_t)(1 + n_d - (MA - 1)) * dm.d;
+            if (!run_adapter(MA, len_A, f, true)) return false;
+            int tk[M_MAX]; float pp[M_MAX];
+            if (!run_head(D.abuf + (size_t)(MA - 1) * dm.d, 1, D.layers[dm.L].g2,
+                          D.dbg_draft + (size_t)n_steps * dm.V, tk, pp)) return false;
+            len_A += MA;
+            dconf[n_steps] = pp[0];
+            n_steps++;
+            if (pg.stop_mode == 1 && pp[0] <= pg.eta) break;                        // drop the low-confidence token
+            dtok[n_d] = tk[0];
+            n_d++;
+            cur = tk[0];
+            if (pg.stop_mode == 0 && pp[0] <= pg.eta) stop_after_shallow = true;    // keep it; its feature is still needed
+        }
+        if (leader()) {
+            State* st = D.st;
+            st->n_d = n_d; st->n_steps = n_steps; st->len_A = len_A; st->pending = 1;
+            for (int i = 0; i < M_MAX; ++i) { st->draft_tok[i] = dtok[i]; st->conf[i] = dconf[i]; }
+            st->draft_steps_total += n_steps; st->drafted_total += n_d;
+        }
+        return true;
+    }
+
+    // Verify pass + prefix accept + rollback (Section 3: discard after the first reject; Figure 2).
+    __device__ bool verify_phase() {
+        const Dims& dm = D.dm;
+        const int M = n_d + 1;
+        for (int i = dm.l; i < dm.L; ++i)
+            if (!run_layer(i, M, P, (i == dm.l) ? D.feat + dm.d : D.h, D.h)) return false;
+        int t[M_MAX]; float pp[M_MAX];
+        if (!run_head(D.h, M, D.g_final, D.dbg_verify, t, pp)) return false;
+        int k = 0;
+        while (k < n_d && dtok[k] == t[k]) ++k;
+        const int newP = P + k + 1;
+        if (len_A > newP) len_A = newP;
+        if (len_A < newP) {
+            // the adapter has not seen f[k] (k == n_d): keep it as the feature of position newP-1
+            const float* src = D.feat + (size_t)(1 + k) * dm.d;
+            for (int e = c.cta * NTHREADS + threadIdx.x; e < dm.d; e += c.nctas * NTHREADS) D.feat[e] = __ldcg(src + e);
+        }
+        if (leader()) {
+            State* st = D.st;
+            for (int i = 0; i < k; ++i) { D.out_tokens[total + i] = dtok[i]; st->emitted[i] = dtok[i]; }
+            D.out_tokens[total + k] = t[k]; st->emitted[k] = t[k];
+            for (int i = 0; i < M; ++i) st->target[i] = t[i];
+            D.S[rounds] = k + 1;
+            D.round_log[rounds * 4 + 0] = n_d; D.round_log[rounds * 4 + 1] = n_steps;
+            D.round_log[rounds * 4 + 2] = k; D.round_log[rounds * 4 + 3] = P;
+            st->M = M; st->k_acc = k; st->n_emit = k + 1;
+            st->P = newP; st->len_A = len_A; st->x0 = t[k]; st->pending = 0;
+            st->total = total + k + 1; st->rounds = rounds + 1; st->accepted_total += k;
+        }
+        P = newP; x0 = t[k]; total += k + 1; rounds += 1;
+        return true;
+    }
+
+    __device__ bool prefill() {
+        const Dims& dm = D.dm;
+        const int n = pg.n;
+        int tk[M_MAX]; float pp[M_MAX];
+        for (int c0 = 0; c0 < n; c0 += M_MAX) {
+            const int M = min(M_MAX, n - c0);
+            embed_rows(D.prompt + c0, 0, M, D.h);
+            KG_SYNC(2);
+            for (int i = 0; i < dm.l; ++i) if (!run_layer(i, M, c0, D.h, D.h)) return false;
+            if (!run_adapter(M, c0, D.h, false)) return false;
+            for (int i = dm.l; i < dm.L; ++i) if (!run_layer(i, M, c0, D.h, D.h)) return false;
+            if (c0 + M == n)
+                if (!run_head(D.h + (size_t)(M - 1) * dm.d, 1, D.g_final, D.dbg_verify, tk, pp)) return false;
+        }
+        if (leader()) {
+            State* st = D.st;
+            st->P = n; st->len_A = n; st->x0 = tk[0]; st->pending = 0; st->total = 1; st->rounds = 0;
+            D.out_tokens[0] = tk[0];
+        }
+        return true;
+    }
+
+    __device__ bool ar_decode() {
+        const Dims& dm = D.dm;
+        int tk[M_MAX]; float pp[M_MAX];
+        while (total < pg.n) {
+            embed_rows(nullptr, x0, 1, D.h);
+            KG_SYNC(3);
+            for (int i = 0; i < dm.L; ++i) if (!run_layer(i, 1, P, D.h, D.h)) return false;
+            if (!run_head(D.h, 1, D.g_final, D.dbg_verify, tk, pp)) return false;
+            if (leader()) {
+                D.out_tokens[total] = tk[0];
+                D.st->P = P + 1; D.st->x0 = tk[0]; D.st->total = total + 1; D.st->len_A = -1;
+            }
+            P += 1; x0 = tk[0]; total += 1;
+        }
+        return true;
+    }
+
+    __device__ void run() {
+        load_state();
+        switch (pg.kind) {
+            case PROG_PREFILL: prefill(); break;
+            case PROG_DRAFT: draft_phase(); break;
+            case PROG_VERIFY: verify_phase(); break;
+            case PROG_AR: ar_decode(); break;
+            case PROG_DECODE:
+                while (total < pg.n) {
+                    if (!draft_phase()) return;
+                    if (!verify_phase()) return;
+                }
+                break;
+        }
+    }
+};
+
+template <typename WT>
+__global__ void __launch_bounds__(NTHREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
+    extern __shared__ __align__(128) char smem[];
+    Ctx c;
+    c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = D.st; c.bar = D.bar; c.smem = smem; c.grid = true;
+    Engine<WT> eng(D, c, pg);
+    eng.run();
+}
+
+}  // namespace kg

@@ -1,0 +1,174 @@
+"""CUDA path vs CPU oracle through the C ABI: bit-exact tokens and accept lengths, logits within
+2e-2, confidences within 1e-3 (tolerances of the benchmark spec), on the tiny fp32 model, small
+bf16 models (tensor-core path, several tiles and ragged tails) and sampled rounds of the 7B shape."""
+import numpy as np
+import pytest
+
+import kg_inputs as ki
+from oracle import kangaroo_oracle as ko
+
+pytestmark = pytest.mark.gpu
+
+TINY = ki.get_config("tiny")
+# bf16 model whose matrices span several 16-row tiles per CTA chunk and ragged K phases
+SMALL_BF = ki.KgShape("small_bf", 3, 512, 4, 128, 1376, 2048, 1, "bf16", logit_scale=10.0, max_seq=160,
+                      page_size=16, gamma_max=10, gain_std=0.1, deep_resid_scale=0.1, adapter_resid_scale=0.1,
+                      n_prompt=21, n_gen=40, seed=5)
+MICRO_BF = ki.KgShape("micro_bf", 2, 64, 2, 32, 96, 128, 1, "bf16", logit_scale=12.0, max_seq=96, page_size=4,
+                      gamma_max=6, gain_std=0.2, deep_resid_scale=0.3, adapter_resid_scale=0.3, n_prompt=9, n_gen=24, seed=3)
+
+
+@pytest.fixture(scope="module")
+def binding():
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_2404_18911_b200 import binding as b
+    b.load()
+    return b
+
+
+def _pair(binding, shape, dtype=np.float64, **kw):
+    g = binding.KangarooModel(shape, debug_logits=True, **kw)
+    o = ko.KangarooOracle(shape, ki.make_weights(shape), dtype)
+    return g, o
+
+
+@pytest.mark.parametrize("shape", [TINY, MICRO_BF, SMALL_BF], ids=lambda s: s.name)
+def test_device_weights_equal_host_generator(binding, shape):
+    g = binding.KangarooModel(shape)
+    w = ki.make_weights(shape, force_numpy=True)
+    L = shape.n_layers
+    checks = [("embed", 0, w["embed"]), ("head", 0, w["head"]), ("g_final", 0, w["g_final"]),
+              ("wqkv", 0, w["layers"][0]["wqkv"]), ("wo", L - 1, w["layers"][L - 1]["wo"]),
+              ("wgate", 1, w["layers"][1]["wgate"]), ("wup", 0, w["layers"][0]["wup"]),
+              ("wdown", L - 1, w["layers"][L - 1]["wdown"]), ("g1", 1, w["layers"][1]["g1"]),
+              ("g2", 0, w["layers"][0]["g2"]), ("wqkv", L, w["adapter"]["wqkv"]), ("wo", L, w["adapter"]["wo"]),
+              ("g1", L, w["adapter"]["g_in"]), ("g2", L, w["adapter"]["g_last"])]
+    for name, layer, ref in checks:
+        ref = ref.reshape(-1)
+        got = g.read_weight(name, layer, 0, ref.size)
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), (name, layer)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("shape", [TINY, MICRO_BF, SMALL_BF], ids=lambda s: s.name)
+def test_lockstep_parity(binding, shape, mode):
+    from parity_harness import lockstep
+    g, o = _pair(binding, shape)
+    prompt = ki.make_prompt(shape).tolist()
+    res = lockstep(g, o, prompt, shape.n_gen, shape.eta, shape.gamma, mode)
+    assert len(res["flips"]) <= 2, res["flips"]
+    assert res["max_logit_err"] < 2e-2 and res["max_conf_err"] < 1e-3
+    assert all(1 <= s <= shape.gamma + 1 for s in res["S"])
+    if not res["flips"]:
+        ar = o.generate_ar(prompt, shape.n_gen)
+        assert res["tokens"][: shape.n_gen] == ar
+
+
+@pytest.mark.parametrize("eta,gamma", [(0.0, 1), (0.0, 6), (0.3, 2), (0.9, 10), (1.5, 3)])
+def test_lockstep_eta_gamma_grid(binding, eta, gamma):
+    from parity_harness import lockstep
+    g, o = _pair(binding, TINY)
+    prompt = ki.make_prompt(TINY).tolist()
+    for mode in (0, 1):
+        res = lockstep(g, o, prompt, 30, eta, gamma, mode)
+        assert not res["flips"]
+        if eta == 0.0:
+            assert all(r["n_drafted"] == gamma for r in o.log)
+        if eta > 1.0:
+            assert all(r["n_drafted"] == (1 if mode == 0 else 0) for r in o.log)
+
+
+def test_page_table_indirection_and_plain_path(binding):
+    """A permuted page table and the plain (non tensor-core) linear path give the same tokens."""
+    shape = SMALL_BF
+    prompt = ki.make_prompt(shape).tolist()
+    g0 = binding.KangarooModel(shape)
+    t0, s0 = g0.generate(prompt, 32, 0.6, 6)
+    g1 = binding.KangarooModel(shape, page_shuffle=True)
+    t1, s1 = g1.generate(prompt, 32, 0.6, 6)
+    assert t0 == t1 and s0["rounds"] == s1["rounds"]
+    g0.force_simple(True)
+    t2, s2 = g0.generate(prompt, 32, 0.6, 6)
+    assert t2 == t0
+
+
+@pytest.mark.parametrize("shape", [TINY, SMALL_BF], ids=lambda s: s.name)
+def test_generate_matches_oracle_and_is_lossless(binding, shape):
+    g, o = _pair(binding, shape)
+    prompt = ki.make_prompt(shape).tolist()
+    n = shape.n_gen
+    toks, st = g.generate(prompt, n, shape.eta, shape.gamma)
+    ref = o.generate(prompt, n, shape.eta, shape.gamma)
+    assert toks == ref
+    assert g.read_S()[: st["rounds"] - 1] == o.S[:-1]
+    assert st["rounds"] == len(o.S) and st["tokens"] == n - 1
+    assert abs(st["cr"] - ko.compression_rate(o.S)) < 1e-12
+    for w_ in range(shape.gamma + 2):
+        assert abs(st["ctar"][w_] - ko.ctar(o.S, w_)) < 1e-12
+    # plain greedy decoding on the GPU gives the same tokens (lossless)
+    g.reset()
+    g.prefill(prompt)
+    assert g.decode_ar(n) == toks
+    # two runs are bit-identical (fixed reduction orders)
+    toks2, _ = g.generate(prompt, n, shape.eta, shape.gamma)
+    assert toks2 == toks
+
+
+def test_microbench_state_verify_matches_oracle(binding):
+    """Verify step on a seeded N(0,1) KV cache and N(0,1) early features (the verify-step
+    microbenchmark's inputs) against the oracle's deep layers on the same inputs."""
+    shape = SMALL_BF
+    T, seed = 77, 11
+    for n_d in (0, 3, 9):
+        g = binding.KangarooModel(shape, debug_logits=True)
+        g.fill_state(T, n_d, seed)
+        v = g.verify()
+        o = ko.KangarooOracle(shape, ki.make_weights(shape))
+        st = ki.microbench_state(shape, T, n_d, seed)
+        for i in range(shape.n_layers):
+            o.cache[i].k[:T], o.cache[i].v[:T], o.cache[i].length = st["k"][i], st["v"][i], T
+        feats = [st["feat"][1 + j].astype(np.float64) for j in range(n_d + 1)]
+        t, z = o._verify_tokens(feats, T)
+        for i in range(n_d + 1):
+            err = float(np.max(np.abs(g.debug_logits(1, i) - z[i])))
+            assert err < 2e-2, (n_d, i, err)
+            assert v["target"][i] == t[i] or ko.top2_gap(z[i]) < 2e-2
+        assert v["n_rows"] == n_d + 1
+
+
+def test_api_errors(binding):
+    b = binding
+    g = b.KangarooModel(TINY)
+    with pytest.raises(b.KgError) as e:
+        g.draft(0.6, 6)
+    assert e.value.status == b.KG_E_STATE                     # draft before prefill
+    g.prefill(ki.make_prompt(TINY).tolist())
+    with pytest.raises(b.KgError) as e:
+        g.verify()
+    assert e.value.status == b.KG_E_STATE                     # verify without a pending draft
+    with pytest.raises(b.KgError) as e:
+        g.draft(0.6, 0)
+    assert e.value.status == b.KG_E_ARG
+    with pytest.raises(b.KgError) as e:
+        g.draft(0.6, TINY.gamma_max + 1)
+    assert e.value.status == b.KG_E_ARG
+    with pytest.raises(b.KgError) as e:
+        g.prefill([1, 2, 3])
+    assert e.value.status == b.KG_E_STATE                     # prefill needs a reset model
+    g.reset()
+    with pytest.raises(b.KgError) as e:
+        g.prefill(list(range(TINY.max_seq + 5)))
+    assert e.value.status == b.KG_E_SEQ_FULL
+    with pytest.raises(b.KgError) as e:
+        g.prefill([TINY.vocab])
+    assert e.value.status == b.KG_E_ARG
+    g.prefill([1, 2, 3])
+    with pytest.raises(b.KgError) as e:
+        g.decode(TINY.max_seq, 0.6, 6)
+    assert e.value.status == b.KG_E_SEQ_FULL
+    g.draft(0.6, 6)
+    with pytest.raises(b.KgError) as e:
+        g.draft(0.6, 6)
+    assert e.value.status == b.KG_E_STATE                     # a draft is already pending
+    g.verify()
