@@ -151,6 +151,11 @@ int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_prompt, int32
 int kg_read_tokens(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out);
 int kg_read_S(kg_model* m, int32_t* out_host, int32_t max_n, int32_t* n_out);
 
+/* Per-round record of the rounds run so far, four int32 per round: n_d (drafts kept), n_steps
+ * (adapter+head passes), k (drafts accepted), P (position of the round's x_0, Figure 2).  Copies at
+ * most max_rounds records to out_host[max_rounds * 4]; synchronises. */
+int kg_read_round_log(kg_model* m, int32_t* out_host, int32_t max_rounds, int32_t* n_out);
+
 /* Parity helpers (need cfg.debug_logits = 1).  which = 0: draft logits of step `row` of the last
  * round; which = 1: verify / AR / prefill logits of row `row` of the last pass.  Copies V floats. */
 int kg_debug_logits(kg_model* m, int32_t which, int32_t row, float* out_host);

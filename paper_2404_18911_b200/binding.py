@@ -21,7 +21,7 @@ KG_OK, KG_E_ARG, KG_E_STATE, KG_E_NOMEM, KG_E_SEQ_FULL, KG_E_CUDA, KG_E_TIMEOUT 
 
 EXPORTS = [
     "kg_workspace_bytes", "kg_init_model", "kg_free_model", "kg_reset", "kg_prefill", "kg_prefill_device",
-    "kg_draft", "kg_verify", "kg_decode", "kg_decode_ar", "kg_generate", "kg_read_tokens", "kg_read_S",
+    "kg_draft", "kg_verify", "kg_decode", "kg_decode_ar", "kg_generate", "kg_read_tokens", "kg_read_S", "kg_read_round_log",
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
     "kg_op_lm_head", "kg_op_attention", "kg_strerror",
 ]
@@ -100,6 +100,7 @@ def load():
     lib.kg_generate.argtypes = [vp, vp, i32, i32, f32, i32, i32, vp, C.POINTER(i32), C.POINTER(KgStats)]
     lib.kg_read_tokens.argtypes = [vp, vp, i32, C.POINTER(i32)]
     lib.kg_read_S.argtypes = [vp, vp, i32, C.POINTER(i32)]
+    lib.kg_read_round_log.argtypes = [vp, vp, i32, C.POINTER(i32)]
     lib.kg_debug_logits.argtypes = [vp, i32, i32, vp]
     lib.kg_read_weight.argtypes = [vp, C.c_char_p, i32, u64, u64, vp]
     lib.kg_debug_fill_state.argtypes = [vp, i32, i32, u64]
@@ -226,6 +227,15 @@ class KangarooModel:
                                     out.ctypes.data, C.byref(n), C.byref(st)), "kg_generate")
         return out[:n.value].tolist(), self._stats(st)
 
+    def generate_into(self, prompt_host, out_host, max_new, eta, gamma, stop_mode=STOP_KEEP):
+        """kg_generate on caller-owned host tensors (e.g. pinned torch int32 tensors): the prompt is read
+        from prompt_host, the tokens are written to out_host.  Returns (n_out, stats)."""
+        n = C.c_int32()
+        st = KgStats()
+        _check(self.lib.kg_generate(self.h, prompt_host.data_ptr(), prompt_host.numel(), max_new, eta, gamma, stop_mode,
+                                    out_host.data_ptr(), C.byref(n), C.byref(st)), "kg_generate")
+        return n.value, self._stats(st)
+
     def read_tokens(self, max_n=None):
         max_n = self.shape.max_seq + KG_M_MAX if max_n is None else max_n
         out = np.empty(max_n, dtype=np.int32)
@@ -239,6 +249,14 @@ class KangarooModel:
         n = C.c_int32()
         _check(self.lib.kg_read_S(self.h, out.ctypes.data, max_n, C.byref(n)), "kg_read_S")
         return out[:n.value].tolist()
+
+    def read_round_log(self, max_rounds=None):
+        """One (n_d, n_steps, k, P) tuple per round run so far."""
+        max_rounds = self.shape.max_seq + KG_M_MAX if max_rounds is None else max_rounds
+        out = np.empty((max_rounds, 4), dtype=np.int32)
+        n = C.c_int32()
+        _check(self.lib.kg_read_round_log(self.h, out.ctypes.data, max_rounds, C.byref(n)), "kg_read_round_log")
+        return [tuple(int(v) for v in row) for row in out[:n.value]]
 
     def debug_logits(self, which, row):
         out = np.empty(self.shape.vocab, dtype=np.float32)

@@ -548,6 +548,20 @@ extern "C" int kg_read_S(kg_model* m, int32_t* out_host, int32_t max_n, int32_t*
     return KG_OK;
 }
 
+extern "C" int kg_read_round_log(kg_model* m, int32_t* out_host, int32_t max_rounds, int32_t* n_out) {
+    if (!m || !out_host || max_rounds < 0) return KG_E_ARG;
+    State st;
+    int r = read_state(m, &st);
+    if (r != KG_OK) return r;
+    const int n = st.rounds < max_rounds ? st.rounds : max_rounds;
+    if (n > 0) {
+        CK(cudaMemcpyAsync(out_host, m->dev.round_log, sizeof(int) * 4 * n, cudaMemcpyDeviceToHost, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+    if (n_out) *n_out = n;
+    return KG_OK;
+}
+
 extern "C" int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_prompt, int32_t max_new,
                            float eta, int32_t gamma, int32_t stop_mode,
                            int32_t* out_tokens_host, int32_t* n_out, kg_stats* stats) {
