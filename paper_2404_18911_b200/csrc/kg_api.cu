@@ -92,8 +92,8 @@ bool valid_config(const kg_config* c) {
     if (c->n_heads > 256) return false;
     // the plain path stages all rows of an operand in shared memory
     const int kmax = c->d_ffn > c->d_model ? c->d_ffn : c->d_model;
-    const bool plain_everywhere = c->dtype == KG_F32 || (c->d_model % 32) || (c->d_ffn % 32);
-    if (plain_everywhere && (size_t)kmax * KG_M_MAX * 4 > (size_t)XS_BUDGET) return false;
+    const bool plain_somewhere = c->dtype == KG_F32 || (c->d_model % 16) || (c->d_ffn % 16);
+    if (plain_somewhere && (size_t)kmax * KG_M_MAX * 4 > (size_t)SIMPLE_XS_BYTES) return false;
     return true;
 }
 
@@ -205,7 +205,7 @@ static int launch_program(kg_model* m, const Program& pg) {
     Program p = pg;
     p.force_simple = m->force_simple;
     void* args[] = {(void*)&m->dev, (void*)&p};
-    CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(NTHREADS), args, m->smem, m->stream));
+    CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(BLOCK_THREADS), args, m->smem, m->stream));
     return KG_OK;
 }
 static int launch(kg_model* m, const Program& pg) {
@@ -273,13 +273,13 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     m->cfg = *cfg; m->lay = lay; m->arena = base; m->stream = (cudaStream_t)cuda_stream; m->nctas = nctas;
     m->own_weights = own != 0; m->prefilled = m->pending = m->ar_used = m->dead = false;
     m->gamma_pending = 0; m->P_upper = 0; m->force_simple = 0;
-    m->smem = smem_bytes_needed();
+    m->smem = SMEM_TOTAL;
 
     const bool bf = cfg->dtype == KG_BF16;
     const void* kfn = bf ? (const void*)kg_persistent_kernel<__nv_bfloat16> : (const void*)kg_persistent_kernel<float>;
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m->smem) != cudaSuccess) { delete m; return KG_E_CUDA; }
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kfn, NTHREADS, m->smem) != cudaSuccess || occ < 1) { delete m; return KG_E_CUDA; }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kfn, BLOCK_THREADS, m->smem) != cudaSuccess || occ < 1) { delete m; return KG_E_CUDA; }
 
     Dev& D = m->dev;
     std::memset(&D, 0, sizeof(D));
@@ -701,26 +701,29 @@ OpScratch op_layout() {
 }
 
 template <typename WT>
-__global__ void __launch_bounds__(NTHREADS, 1) op_linear_kernel(LinArgs a, State* st, int force_simple) {
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int force_simple) {
     extern __shared__ __align__(128) char smem[];
-    Ctx c; c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = nullptr; c.smem = smem; c.grid = false;
-    LinDispatch<WT>::run(a, c, force_simple != 0);
+    Ctx c;
+    ctx_init(c, smem, nullptr, nullptr, false);
+    const bool ok = linear_op<WT>(a, c, force_simple != 0);
+    if (!ok && c.producer) ring_drain(c);
 }
 __global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* tok, float* p) {
     if (threadIdx.x < M) { int t; float pp; head_final(part, nctas, threadIdx.x, t, pp); tok[threadIdx.x] = t; p[threadIdx.x] = pp; }
 }
 template <typename WT>
-__global__ void __launch_bounds__(NTHREADS, 1) op_attention_kernel(const __grid_constant__ Dev D, AttArgs a) {
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_attention_kernel(const __grid_constant__ Dev D, AttArgs a) {
     extern __shared__ __align__(128) char smem[];
-    Ctx c; c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = nullptr; c.bar = nullptr; c.smem = smem; c.grid = false;
-    attention_op<WT>(D, a, c);
+    Ctx c;
+    ctx_init(c, smem, nullptr, nullptr, false);
+    if (!c.producer) attention_op<WT>(D, a, c);
 }
 
 int g_force_simple_ops = 0;
 
 template <typename K>
 int set_smem(K kfn) {
-    return cudaFuncSetAttribute((const void*)kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_needed()) == cudaSuccess ? KG_OK : KG_E_CUDA;
+    return cudaFuncSetAttribute((const void*)kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL) == cudaSuccess ? KG_OK : KG_E_CUDA;
 }
 
 }  // namespace
@@ -732,15 +735,15 @@ extern "C" int kg_debug_force_simple_ops(int on) { g_force_simple_ops = on ? 1 :
 static int op_linear_common(int32_t dtype, LinArgs& a, cudaStream_t s) {
     if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
     if (a.M < 1 || a.M > KG_M_MAX || a.N < 1 || a.K < 8 || (a.K % 8)) return KG_E_ARG;
-    const bool plain = dtype == KG_F32 || g_force_simple_ops || (a.K % 32);
-    if (plain && (size_t)a.K * a.M * 4 > (size_t)XS_BUDGET) return KG_E_ARG;
+    const bool plain = dtype == KG_F32 || g_force_simple_ops || (a.K % 16);
+    if (plain && (size_t)a.K * a.M * 4 > (size_t)SIMPLE_XS_BYTES) return KG_E_ARG;
     const int nctas = sm_count();
     if (dtype == KG_BF16) {
         if (set_smem(op_linear_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<__nv_bfloat16><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(a, nullptr, g_force_simple_ops);
+        op_linear_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, g_force_simple_ops);
     } else {
         if (set_smem(op_linear_kernel<float>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<float><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(a, nullptr, g_force_simple_ops);
+        op_linear_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, g_force_simple_ops);
     }
     CK(cudaGetLastError());
     return KG_OK;
@@ -796,10 +799,10 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
     const int nctas = sm_count();
     if (dtype == KG_BF16) {
         if (set_smem(op_attention_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
-        op_attention_kernel<__nv_bfloat16><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(D, a);
+        op_attention_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, a);
     } else {
         if (set_smem(op_attention_kernel<float>) != KG_OK) return KG_E_CUDA;
-        op_attention_kernel<float><<<nctas, NTHREADS, smem_bytes_needed(), s>>>(D, a);
+        op_attention_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, a);
     }
     CK(cudaGetLastError());
     return KG_OK;

@@ -5,26 +5,51 @@
 // (cta, nctas) and a grid-wide barrier separates dependent operators.  The same operators are
 // also wrapped one-by-one in small kernels for unit tests.
 //
-// Data flow is weight streaming: every weight byte is read exactly once per pass, straight from
-// HBM into registers with 128-bit non-allocating loads, and consumed by tensor-core MMAs whose
-// "M" side is the weight tile and whose "N" side is the 1..16 activation rows.
+// A CTA has 16 consumer warps and one producer warp.  The decode step is bound by HBM bandwidth:
+// every weight byte is read exactly once per pass.  The producer warp streams this CTA's share of
+// every weight matrix of a pass through a ring of shared-memory slots with bulk asynchronous
+// copies (cp.async.bulk + mbarrier transaction counts); because weights do not depend on
+// activations it runs ahead of the consumers across operator boundaries and grid barriers, so HBM
+// stays busy while the consumers synchronise.  The consumers read weight tiles with ldmatrix and
+// feed tensor-core MMAs whose "M" side is the weight tile and whose "N" side is the 1..16
+// activation rows (activations split into bf16 hi + lo so that the product keeps fp32 accuracy).
 #pragma once
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Timeline hook for profiling builds (a translation unit may define it before including this file).
+#ifndef KG_PROBE
+#define KG_PROBE(slot) do { } while (0)
+#endif
+
 namespace kg {
 
 constexpr int M_MAX = 16;          // rows per pass
-constexpr int NTHREADS = 512;      // threads per CTA
+constexpr int NTHREADS = 256;      // consumer threads per CTA
 constexpr int NWARPS = NTHREADS / 32;
+constexpr int BLOCK_THREADS = NTHREADS + 32;   // + the producer warp (warp index NWARPS)
 constexpr int S_CAP = 16;          // most KV splits per head
 constexpr int ATT_TK = 64;         // keys per attention tile
 constexpr int HD_MAX = 128;
-constexpr int LIN_U = 4;           // k32-steps in flight per warp iteration
-constexpr int XS_BUDGET = 168 * 1024;   // shared-memory bytes for staged activations
-constexpr unsigned long long BARRIER_TIMEOUT_CLK = 6000000000ull;   // ~3 s at 1.9 GHz
+
+// weight ring: RING slots of ST_ROWS weight rows x ST_K k-elements (bf16); rows are padded by 16
+// bytes so that the eight row addresses of an ldmatrix fall into distinct bank groups
+constexpr int RING = 4;
+constexpr int ST_ROWS = 8;
+constexpr int ST_K = 2048;
+constexpr int ST_ROW_BYTES = ST_K * 2 + 16;
+constexpr int SLOT_BYTES = ST_ROWS * ST_ROW_BYTES;
+constexpr int CTRL_BYTES = 1024;
+constexpr int RING_OFF = CTRL_BYTES;
+constexpr int WORK_OFF = RING_OFF + RING * SLOT_BYTES;
+constexpr int SMEM_TOTAL = 232448;                      // 227 KB, the most one CTA may own
+constexpr int WORK_BYTES = SMEM_TOTAL - WORK_OFF;       // activations, reductions, attention tiles
+constexpr int SC_ROWS = 256;                            // rows whose accumulators live in shared memory at once
+constexpr int SIMPLE_XS_BYTES = WORK_BYTES - 4096;      // activation staging of the plain path
+
+constexpr unsigned long long WAIT_TIMEOUT_CLK = 6000000000ull;   // ~3 s at 1.9 GHz
 
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_HEAD = 3 };
 enum { ST_OK = 0, ST_TIMEOUT = -6 };
@@ -84,35 +109,101 @@ struct Dev {
     double inv_freq[HD_MAX / 2];   // theta^(-2i/hd)
 };
 
+// Per-CTA control block at the start of shared memory.
+struct Ctrl {
+    unsigned long long full[RING];     // producer -> consumers: slot filled (transaction count)
+    unsigned long long empty[RING];    // consumers -> producer: slot drained (one arrival per consumer warp)
+    unsigned long long mail;           // consumers -> producer: head_tok / head_p hold a new result
+    unsigned long long xfull;          // activation rows of a k phase have landed in shared memory
+    int abort;                         // a bounded wait of this CTA gave up
+    int sync_ok;
+    int att_last;
+    int head_tok[M_MAX];
+    float head_p[M_MAX];
+};
+static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+
 struct Ctx {
     int cta, nctas;
-    unsigned bar_target;           // arrivals expected at the next barrier (thread 0 only)
+    unsigned bar_target;           // arrivals expected at the next grid barrier (thread 0 only)
     State* st; unsigned* bar;
     char* smem;
-    bool grid;                     // false: single-operator test kernel, barriers are no-ops
+    Ctrl* ctl;
+    bool grid;                     // false: single-operator test kernel, grid barriers are CTA barriers
+    bool producer;                 // this thread belongs to the producer warp
+    int slot; unsigned phase;      // ring cursor of this thread's role
+    unsigned issued;               // producer: stages issued so far
+    unsigned mail_phase;           // producer: parity of the next result it waits for
+    unsigned x_phase;              // consumers: parity of the next activation stage
 };
 
 // ------------------------------------------------------------------------------------ helpers
 
-__device__ __forceinline__ uint4 ldg_stream16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ float2 ldcg_f2(const float* p) { return __ldcg(reinterpret_cast<const float2*>(p)); }
 __device__ __forceinline__ float4 ldcg_f4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
-                                               unsigned b0, unsigned b1) {
+// barrier among the consumer warps only (the producer warp never takes part)
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory"); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// global -> shared bulk copy; bytes and both addresses are multiples of 16
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsigned bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void record_timeout(Ctx& c, int where) {
+    *(volatile int*)&c.ctl->abort = 1;
+    if (c.st) {
+        atomicCAS(&c.st->status, 0, ST_TIMEOUT);
+        c.st->timeout_where = where;
+    }
+}
+
+// Bounded wait on an mbarrier phase.  Returns false when this CTA has given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(Ctx& c, unsigned long long* bar, unsigned parity, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if (((++spins) & 63u) == 0u) {
+            if (*(volatile int*)&c.ctl->abort) return false;
+            if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); return false; }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -146,13 +237,31 @@ __device__ __forceinline__ bool arg_better(float za, int ia, float zb, int ib) {
     return za > zb || (za == zb && ia < ib);
 }
 
-// ------------------------------------------------------------------------------------ grid barrier
-// Monotonic arrival counter; every wait is bounded.  On expiry the kernel records KG_E_TIMEOUT in
-// the state word and every CTA leaves at its next barrier.  Returns false when the grid must stop.
-__device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
-    if (!c.grid) { __syncthreads(); return true; }
-    __shared__ int s_ok;
+// ------------------------------------------------------------------------------------ CTA set-up
+// Called by every thread of the CTA at kernel start.
+__device__ __forceinline__ void ctx_init(Ctx& c, char* smem, State* st, unsigned* bar, bool grid) {
+    c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
+    c.ctl = reinterpret_cast<Ctrl*>(smem); c.grid = grid;
+    c.producer = threadIdx.x >= NTHREADS;
+    c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0; c.x_phase = 0;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < RING; ++i) { mbar_init(&c.ctl->full[i], 1); mbar_init(&c.ctl->empty[i], NWARPS); }
+        mbar_init(&c.ctl->mail, 1);
+        mbar_init(&c.ctl->xfull, 1);
+        c.ctl->abort = 0; c.ctl->sync_ok = 1; c.ctl->att_last = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------ grid barrier
+// Consumer threads only.  Monotonic arrival counter; every wait is bounded.  On expiry the kernel
+// records KG_E_TIMEOUT in the state word and every CTA leaves at its next barrier.  Returns false
+// when the grid must stop (the same value in every consumer thread of the CTA).
+__device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
+    if (!c.grid) { cta_sync(); return *(volatile int*)&c.ctl->abort == 0; }
+    cta_sync();
+    KG_PROBE(1);
     if (threadIdx.x == 0) {
         c.bar_target += (unsigned)c.nctas;
         __threadfence();
@@ -163,18 +272,16 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
         while ((int)(ld_acquire_u32(c.bar) - c.bar_target) < 0) {
             if (((++spins) & 63u) == 0u) {
                 if (*(volatile int*)&c.st->status != 0) { ok = 0; break; }
-                if ((unsigned long long)(clock64() - t0) > BARRIER_TIMEOUT_CLK) {
-                    atomicCAS(&c.st->status, 0, ST_TIMEOUT);
-                    c.st->timeout_where = where;
-                    ok = 0;
-                    break;
-                }
+                if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
             }
         }
-        s_ok = ok;
+        if (*(volatile int*)&c.st->status != 0) ok = 0;
+        if (!ok) *(volatile int*)&c.ctl->abort = 1;          // lets the producer warp leave its waits
+        c.ctl->sync_ok = ok;
     }
-    __syncthreads();
-    return s_ok != 0;
+    cta_sync();
+    KG_PROBE(2);
+    return *(volatile int*)&c.ctl->sync_ok != 0;
 }
 
 // ------------------------------------------------------------------------------------ RoPE
@@ -217,152 +324,280 @@ __device__ __forceinline__ void head_merge(HeadStat& a, float zmax, float sum, i
     }
 }
 
-// Tensor-core path, bf16 weights, 1 <= M <= 8*NT.  Swap-AB: the weight tile is the 16-row MMA
-// operand, the activation rows are the 8 MMA columns.  A fragments come straight from global
-// memory: lane (g, t) loads 16 contiguous bytes of weight row g and of row g+8; the k index is
-// permuted identically for A and B so no shuffle or shared-memory staging of weights is needed.
-// Activations are staged once per CTA in shared memory as bf16 hi + lo (x = hi + lo to ~2^-17),
-// with the RMSNorm gain folded in; the 1/rms factor is applied in the epilogue.
-template <int NT>
-__device__ void lin_mma(const LinArgs& a, Ctx& c) {
+// ---- streamed tensor-core path (bf16 weights, K a multiple of 16) -----------------------------------
+//
+// Work split.  The CTA owns a contiguous range of "units": output rows, or for the SwiGLU pair
+// gate/up feature pairs.  A stage of the ring holds 8 weight rows (for the pair: the 8 gate rows of
+// a feature group, then in the next stage the 8 up rows of the same features) times one k phase
+// (2048 k-elements when M <= 8, else 1024), i.e. one bulk copy of up to 4 KB per row: the copy
+// engine spends a fixed time per copy, and only copies of 2-4 KB and more keep HBM saturated.
+// The stages are visited superchunk (<= 256 accumulator rows) -> phase -> row group, in the same
+// order by the producer warp (which issues the copies) and the consumers.
+//
+// Consumers take the stages two at a time: one MMA m16n8k16 computes D[weight row, activation
+// column] with the 16 weight rows of a stage pair as the A operand (ldmatrix straight from the
+// ring) and the activations as the 8-column B operand.  The activations keep fp32 accuracy by a
+// split x * gain = hi + lo into two bf16 parts:
+//   V = 4  (M <= 4):  columns 0-3 carry hi, columns 4-7 lo of rows 0-3: one MMA per k16-step;
+//   V = 8  (M <= 8):  hi and lo are two MMAs;
+//   V = 16 (M <= 16): two column tiles, hi and lo: four MMAs.
+// Each of the 8 warps owns a fixed slice of the phase's k range; its B fragments are built once
+// per phase (from an fp32 copy of the activation rows that a bulk copy placed in shared memory one
+// phase ahead) and stay in registers for every row group, so the steady state touches shared
+// memory only for the weights.  After a stage pair the 8 partial sums of each (weight row,
+// activation row) are added in warp order into the per-row accumulators in shared memory.
+template <int V> struct LinGeom {
+    static constexpr int NS = V == 16 ? 8 : 16;           // k16-steps per warp and stage
+    static constexpr int PLEN = NS * 16 * NWARPS;         // k-elements per phase: 2048 or 1024
+    static constexpr int FR = V == 4 ? 2 : (V == 8 ? 4 : 8);   // B fragment registers per step
+    static constexpr int NACC = V == 16 ? 2 : 1;          // column tiles
+};
+constexpr int MP = 16;                                    // accumulator columns (activation rows, padded)
+
+struct LinPlan {
+    int u0, u1;          // this CTA's units
+    int sc_units;        // units per superchunk
+    int plen, nph;       // k phases
+};
+
+__device__ __forceinline__ LinPlan make_plan(const LinArgs& a, int cta, int nctas) {
+    LinPlan p;
+    p.u0 = (int)((long long)a.N * cta / nctas);
+    p.u1 = (int)((long long)a.N * (cta + 1) / nctas);
+    p.sc_units = a.W2 ? SC_ROWS / 2 : SC_ROWS;
+    p.plen = a.M <= 8 ? LinGeom<8>::PLEN : LinGeom<16>::PLEN;
+    p.nph = (a.K + p.plen - 1) / p.plen;
+    return p;
+}
+
+// Producer warp: issue the bulk copies of every stage of this operator.
+__device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
+    const int lane = threadIdx.x & 31;
+    const LinPlan pl = make_plan(a, c.cta, c.nctas);
+    const bool dual = a.W2 != nullptr;
+    const __nv_bfloat16* W = reinterpret_cast<const __nv_bfloat16*>(a.W);
+    const __nv_bfloat16* W2 = reinterpret_cast<const __nv_bfloat16*>(a.W2);
+    char* ring = c.smem + RING_OFF;
+    for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
+        const int sc1 = min(pl.u1, sc0 + pl.sc_units);
+        const int ngrp = (sc1 - sc0 + ST_ROWS - 1) / ST_ROWS;
+        const int nst = dual ? 2 * ngrp : ngrp;
+        for (int ph = 0; ph < pl.nph; ++ph) {
+            const int p0 = ph * pl.plen, len = min(pl.plen, a.K - p0);
+            for (int si = 0; si < nst; ++si) {
+                const int base = sc0 + (dual ? si >> 1 : si) * ST_ROWS;
+                const int nvalid = min(ST_ROWS, sc1 - base);
+                const __nv_bfloat16* src = ((dual && (si & 1)) ? W2 : W) + (size_t)(base + lane) * a.K + p0;
+                int ok = 1;
+                if (lane == 0) ok = mbar_wait(c, &c.ctl->empty[c.slot], c.phase ^ 1u, 40) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) return false;
+                if (lane == 0) mbar_arrive_expect_tx(&c.ctl->full[c.slot], (unsigned)(nvalid * len * 2));
+                __syncwarp();
+                if (lane < nvalid) bulk_g2s(ring + (size_t)c.slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &c.ctl->full[c.slot]);
+                KG_PROBE(30);
+                c.issued++;
+                if (++c.slot == RING) { c.slot = 0; c.phase ^= 1u; }
+            }
+        }
+    }
+    return true;
+}
+
+// Producer warp, after a failed wait: let the copies it still has in flight land before the CTA exits.
+__device__ void ring_drain(Ctx& c) {
+    if ((threadIdx.x & 31) != 0) return;
+    const unsigned n = c.issued < (unsigned)RING ? c.issued : (unsigned)RING;
+    int s = c.slot; unsigned ph = c.phase;
+    for (unsigned i = 0; i < n; ++i) {
+        if (--s < 0) { s = RING - 1; ph ^= 1u; }
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&c.ctl->full[s], ph)) {
+            if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) break;
+        }
+    }
+}
+
+__device__ __forceinline__ void split_hi_lo(float2 v, unsigned& hi, unsigned& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(v.x, v.y);
+    const float2 f = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(v.x - f.x, v.y - f.y);
+    hi = *reinterpret_cast<const unsigned*>(&h);
+    lo = *reinterpret_cast<const unsigned*>(&l);
+}
+
+// Consumer warp 0: start the bulk copies of the activation rows (and the gain) of one k phase.
+__device__ __forceinline__ void issue_x_phase(const LinArgs& a, Ctx& c, char* xs, int p0, int len, int xrow_bytes, int gain_row) {
+    const int lane = threadIdx.x & 31;
+    const int nrows = a.M + (a.gain ? 1 : 0);
+    if (lane == 0) mbar_arrive_expect_tx(&c.ctl->xfull, (unsigned)(nrows * len * 4));
+    asm volatile("fence.proxy.async;" ::: "memory");     // the rows were written with ordinary stores
+    __syncwarp();
+    if (lane < a.M) bulk_g2s(xs + (size_t)lane * xrow_bytes, a.x + (size_t)lane * a.ldx + p0, (unsigned)(len * 4), &c.ctl->xfull);
+    if (lane == M_MAX && a.gain) bulk_g2s(xs + (size_t)gain_row * xrow_bytes, a.gain + p0, (unsigned)(len * 4), &c.ctl->xfull);
+}
+
+template <int V>
+__device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
+    using G = LinGeom<V>;
+    constexpr int NS = G::NS, FR = G::FR, NACC = G::NACC;
+    constexpr int XRB = G::PLEN * 4 + 32;                                  // byte stride of a staged activation row
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int M = a.M, K = a.K;
-    const __nv_bfloat16* W = reinterpret_cast<const __nv_bfloat16*>(a.W);
-    const __nv_bfloat16* W2 = reinterpret_cast<const __nv_bfloat16*>(a.W2);
-    const bool dual = W2 != nullptr;
+    const bool dual = a.W2 != nullptr;
+    const LinPlan pl = make_plan(a, c.cta, c.nctas);
 
-    const long long r0 = (long long)a.N * c.cta / c.nctas;
-    const long long r1 = (long long)a.N * (c.cta + 1) / c.nctas;
-    const int nr = (int)(r1 - r0);
-    const int rpt = dual ? 8 : 16;                       // output rows (or gate/up pairs) per tile
-    const int ntiles = (nr + rpt - 1) / rpt;
-    const int nchunks = (ntiles + 3) / 4;
+    char* xs = c.smem + WORK_OFF;                                          // [V + 1][XRB] fp32 activation rows of a phase, then the gain
+    float* red = reinterpret_cast<float*>(xs + (V + 1) * XRB);             // [2 | 1][NWARPS][NACC][16][8] partial sums
+    float* acc_s = red + 2 * NWARPS * 128;                                 // [SC_ROWS][MP]
+    float* ssw = acc_s + SC_ROWS * MP;                                     // [NWARPS][M_MAX] sums of squares
+    float* rs = ssw + NWARPS * M_MAX;                                      // [M_MAX] 1/rms
+    const char* ring = c.smem + RING_OFF;
 
-    // phases over K so that the staged activations fit
-    int plen_max = (XS_BUDGET / (4 * M) - 32) & ~63;
-    int nph = (K + plen_max - 1) / plen_max;
-    int plen = (((K + nph - 1) / nph) + 63) & ~63;
-    const int xstride = plen + 32;                       // bf16 elements; byte stride = 64 (mod 128)
-
-    __nv_bfloat16* xs_hi = reinterpret_cast<__nv_bfloat16*>(c.smem);
-    __nv_bfloat16* xs_lo = xs_hi + (size_t)M * xstride;
-    float* red = reinterpret_cast<float*>(c.smem + XS_BUDGET);          // [2][NWARPS][NT][16][8]
-    float* ssw = red + 2 * NWARPS * NT * 128;                           // [NWARPS][M_MAX]
-    float* rs = ssw + NWARPS * M_MAX;                                   // [M_MAX]
-
-    for (int i = tid; i < NWARPS * M_MAX; i += NTHREADS) ssw[i] = 0.0f;
-    __syncthreads();
-
-    HeadStat hs; hs.zmax = 0.f; hs.sum = 0.f; hs.arg = 0;               // EPI_HEAD: warp m tracks row m
+    HeadStat hs[2];                                                        // EPI_HEAD: this warp tracks rows warp, warp + 8
+    hs[0].zmax = hs[1].zmax = 0.f; hs[0].sum = hs[1].sum = 0.f; hs[0].arg = hs[1].arg = 0;
+    bool ok = true;
     int buf = 0;
-    bool rs_ready = false;
-
-    for (int ch = 0; ch < nchunks; ++ch) {
-        const int t0 = ch * 4;
-        const int nt = min(4, ntiles - t0);
-        const int n_ks = NWARPS / nt;
-        const int my_tile = warp / n_ks, my_ks = warp % n_ks;
-        const bool active = my_tile < nt;
-        const __nv_bfloat16 *pA = nullptr, *pB = nullptr;
-        if (active) {
-            if (!dual) {
-                long long ra = r0 + (long long)(t0 + my_tile) * 16 + g;
-                if (ra < r1) pA = W + ra * K;
-                if (ra + 8 < r1) pB = W + (ra + 8) * K;
-            } else {
-                long long f = r0 + (long long)(t0 + my_tile) * 8 + g;
-                if (f < r1) { pA = W + f * K; pB = W2 + f * K; }
-            }
-        }
-        float acc[NT][4];
+    KG_PROBE(10);
+    // activation row(s) this lane converts: V = 4: row g & 3 (hi for g < 4, lo otherwise); else rows g (and g + 8)
+    const int xrow = V == 4 ? (g & 3) : g;
+    float ssq[NACC];
 #pragma unroll
-        for (int n = 0; n < NT; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+    for (int n = 0; n < NACC; ++n) ssq[n] = 0.f;
 
-        for (int ph = 0; ph < nph; ++ph) {
-            const int p0 = ph * plen;
-            const int len = min(plen, K - p0);
-            if (nph > 1 || ch == 0) {
-                if (nph > 1) __syncthreads();
-                // stage x[:, p0:p0+len] * gain as bf16 hi / lo; accumulate sum of squares (first chunk only)
-                for (int m = 0; m < M; ++m) {
-                    float ss = 0.f;
-                    const float* xr = a.x + (size_t)m * a.ldx + p0;
-                    for (int u = tid; u < len / 8; u += NTHREADS) {
-                        float4 v0 = ldcg_f4(xr + u * 8), v1 = ldcg_f4(xr + u * 8 + 4);
-                        if (a.gain) {
-                            ss += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w
-                                + v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;
-                            float4 g0 = ldcg_f4(a.gain + p0 + u * 8), g1 = ldcg_f4(a.gain + p0 + u * 8 + 4);
-                            v0.x *= g0.x; v0.y *= g0.y; v0.z *= g0.z; v0.w *= g0.w;
-                            v1.x *= g1.x; v1.y *= g1.y; v1.z *= g1.z; v1.w *= g1.w;
-                        }
-                        float f[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                        __align__(16) __nv_bfloat16 hi[8], lo[8];
+    for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
+        const int sc1 = min(pl.u1, sc0 + pl.sc_units);
+        const int nu = sc1 - sc0;
+        const int ngrp = (nu + ST_ROWS - 1) / ST_ROWS;
+        const int nst = dual ? 2 * ngrp : ngrp;
+        if (warp == 0) issue_x_phase(a, c, xs, 0, min(pl.plen, K), XRB, V);
+        for (int ph = 0; ph < pl.nph; ++ph) {
+            const int p0 = ph * pl.plen, len = min(pl.plen, K - p0);
+            const int nsteps = len / 16;
+            // ---- B fragments of this warp's k slice: x * gain split into bf16 hi / lo
+            unsigned fr[NS][FR];
+            if (ok) ok = mbar_wait(c, &c.ctl->xfull, c.x_phase, 43);
+            c.x_phase ^= 1u;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            hi[e] = __float2bfloat16_rn(f[e]);
-                            lo[e] = __float2bfloat16_rn(f[e] - __bfloat162float(hi[e]));
-                        }
-                        *reinterpret_cast<uint4*>(xs_hi + (size_t)m * xstride + u * 8) = *reinterpret_cast<uint4*>(hi);
-                        *reinterpret_cast<uint4*>(xs_lo + (size_t)m * xstride + u * 8) = *reinterpret_cast<uint4*>(lo);
+            for (int s = 0; s < NS; ++s) {
+#pragma unroll
+                for (int q = 0; q < FR; ++q) fr[s][q] = 0u;
+                const int st = warp * NS + s;
+                if (ok && st < nsteps) {
+                    const int kk = st * 16 + 2 * t;
+                    float2 g0 = make_float2(1.f, 1.f), g1 = g0;
+                    if (a.gain) {
+                        const float* gr = reinterpret_cast<const float*>(xs + (size_t)V * XRB) + kk;
+                        g0 = *reinterpret_cast<const float2*>(gr); g1 = *reinterpret_cast<const float2*>(gr + 8);
                     }
-                    if (a.gain && ch == 0) {
-                        ss = warp_sum(ss);
-                        if (lane == 0) ssw[warp * M_MAX + m] += ss;
+#pragma unroll
+                    for (int n = 0; n < NACC; ++n) {
+                        const int m = xrow + 8 * n;
+                        if (m < M) {
+                            const float* xr = reinterpret_cast<const float*>(xs + (size_t)m * XRB) + kk;
+                            float2 u = *reinterpret_cast<const float2*>(xr), w = *reinterpret_cast<const float2*>(xr + 8);
+                            if (sc0 == pl.u0 && (V != 4 || g < 4)) ssq[n] += u.x * u.x + u.y * u.y + w.x * w.x + w.y * w.y;
+                            u.x *= g0.x; u.y *= g0.y; w.x *= g1.x; w.y *= g1.y;
+                            unsigned h0, l0, h8, l8;
+                            split_hi_lo(u, h0, l0);
+                            split_hi_lo(w, h8, l8);
+                            if (V == 4) { fr[s][0] = g < 4 ? h0 : l0; fr[s][1] = g < 4 ? h8 : l8; }
+                            else { fr[s][4 * n + 0] = h0; fr[s][4 * n + 1] = h8; fr[s][4 * n + 2] = l0; fr[s][4 * n + 3] = l8; }
+                        }
                     }
                 }
-                __syncthreads();
             }
-            if (active) {
-                const int steps = len / 32;
-                const int sb = steps * my_ks / n_ks, se = steps * (my_ks + 1) / n_ks;
-                for (int s = sb; s < se; s += LIN_U) {
-                    uint4 wa[LIN_U], wb[LIN_U];
+            cta_sync();                                      // every warp has read the staged rows
+            if (warp == 0 && ph + 1 < pl.nph) issue_x_phase(a, c, xs, p0 + pl.plen, min(pl.plen, K - p0 - pl.plen), XRB, V);
+            KG_PROBE(11);
+            // ---- the row groups of this phase, two stages (16 weight rows) at a time
+            const uint32_t a_lane = (uint32_t)((lane & 7) * ST_ROW_BYTES + (warp * NS * 16 + (lane >> 4) * 8) * 2);
+            for (int si = 0; si < nst; si += 2) {
+                const bool two = si + 1 < nst;
+                const int slot_a = c.slot;
+                const int slot_b = two ? (slot_a + 1 == RING ? 0 : slot_a + 1) : slot_a;
+                const unsigned phase_b = (two && slot_a + 1 == RING) ? c.phase ^ 1u : c.phase;
+                float acc[4][4];
 #pragma unroll
-                    for (int u = 0; u < LIN_U; ++u) {
-                        wa[u] = make_uint4(0, 0, 0, 0); wb[u] = make_uint4(0, 0, 0, 0);
-                        if (s + u < se) {
-                            const int k = p0 + (s + u) * 32 + 8 * t;
-                            if (pA) wa[u] = ldg_stream16(pA + k);
-                            if (pB) wb[u] = ldg_stream16(pB + k);
-                        }
-                    }
+                for (int q = 0; q < 4; ++q) { acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f; }
+                if (ok) ok = mbar_wait(c, &c.ctl->full[slot_a], c.phase, 41);
+                if (ok && two) ok = mbar_wait(c, &c.ctl->full[slot_b], phase_b, 41);
+                KG_PROBE(12);
+                if (ok) {
+                    // ldmatrix x4: matrices 0, 2 = rows 0-7 (first stage), 1, 3 = rows 8-15 (second stage); k halves 0-7 | 8-15
+                    const uint32_t a_base = smem_u32(ring + (size_t)((lane & 8) ? slot_b : slot_a) * SLOT_BYTES) + a_lane;
 #pragma unroll
-                    for (int u = 0; u < LIN_U; ++u) {
-                        if (s + u < se) {
-                            const int kl = (s + u) * 32 + 8 * t;
-#pragma unroll
-                            for (int n = 0; n < NT; ++n) {
-                                const int m = g + 8 * n;
-                                uint4 xh = make_uint4(0, 0, 0, 0), xl = make_uint4(0, 0, 0, 0);
-                                if (m < M) {
-                                    xh = *reinterpret_cast<const uint4*>(xs_hi + (size_t)m * xstride + kl);
-                                    xl = *reinterpret_cast<const uint4*>(xs_lo + (size_t)m * xstride + kl);
-                                }
-                                mma_bf16_16816(acc[n], wa[u].x, wb[u].x, wa[u].y, wb[u].y, xh.x, xh.y);
-                                mma_bf16_16816(acc[n], wa[u].z, wb[u].z, wa[u].w, wb[u].w, xh.z, xh.w);
-                                mma_bf16_16816(acc[n], wa[u].x, wb[u].x, wa[u].y, wb[u].y, xl.x, xl.y);
-                                mma_bf16_16816(acc[n], wa[u].z, wb[u].z, wa[u].w, wb[u].w, xl.z, xl.w);
+                    for (int s = 0; s < NS; ++s) {
+                        if (warp * NS + s < nsteps) {
+                            unsigned af[4];
+                            ldmatrix_x4(af, a_base + (uint32_t)s * 32u);
+                            if (V == 4) {
+                                mma_bf16_16816(acc[s & 3], af, fr[s][0], fr[s][1]);
+                            } else if (V == 8) {
+                                mma_bf16_16816(acc[(s & 1) * 2], af, fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[(s & 1) * 2 + 1], af, fr[s][2], fr[s][3]);
+                            } else {
+                                mma_bf16_16816(acc[0], af, fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[1], af, fr[s][2], fr[s][3]);
+                                mma_bf16_16816(acc[2], af, fr[s][FR - 4], fr[s][FR - 3]);
+                                mma_bf16_16816(acc[3], af, fr[s][FR - 2], fr[s][FR - 1]);
                             }
                         }
                     }
                 }
-            }
-        }
-        // partial sums of this (tile, k-slice) item
-        float* rb = red + (size_t)buf * NWARPS * NT * 128;
-        if (active) {
+                __syncwarp();
+                KG_PROBE(13);
+                if (ok && lane == 0) { mbar_arrive(&c.ctl->empty[slot_a]); if (two) mbar_arrive(&c.ctl->empty[slot_b]); }
+                c.slot = slot_b; c.phase = phase_b;
+                if (++c.slot == RING) { c.slot = 0; c.phase ^= 1u; }
+                // ---- add the k-slices in warp order into the row accumulators
+                if (V == 16) cta_sync();                     // single partial-sum buffer: the previous pair's sums have been read
+                float* r = red + (size_t)(V == 16 ? 0 : buf) * NWARPS * 128 + (size_t)warp * NACC * 128;
+                if (V == 16) {
+                    // acc[0] / acc[1]: hi / lo of columns 0-7; acc[2] / acc[3]: hi / lo of columns 8-15
+                    *reinterpret_cast<float2*>(r + g * 8 + 2 * t) = make_float2(acc[0][0] + acc[1][0], acc[0][1] + acc[1][1]);
+                    *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) = make_float2(acc[0][2] + acc[1][2], acc[0][3] + acc[1][3]);
+                    *reinterpret_cast<float2*>(r + 128 + g * 8 + 2 * t) = make_float2(acc[2][0] + acc[3][0], acc[2][1] + acc[3][1]);
+                    *reinterpret_cast<float2*>(r + 128 + (g + 8) * 8 + 2 * t) = make_float2(acc[2][2] + acc[3][2], acc[2][3] + acc[3][3]);
+                } else {
+                    *reinterpret_cast<float2*>(r + g * 8 + 2 * t) =
+                        make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
+                    *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) =
+                        make_float2((acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]), (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]));
+                }
+                cta_sync();
+                {
+                    // element (weight row r16, activation row m) of the pair
+                    constexpr int NEL = V == 4 ? 64 : (V == 8 ? 128 : 256);
+                    if (tid < NEL) {
+                        const int r16 = V == 4 ? tid >> 2 : (V == 8 ? tid >> 3 : tid >> 4);
+                        const int m = V == 4 ? tid & 3 : (V == 8 ? tid & 7 : tid & 15);
+                        const float* rb = red + (size_t)(V == 16 ? 0 : buf) * NWARPS * 128 + (V == 16 ? (m >> 3) * 128 : 0) + r16 * 8 + (m & 7);
+                        float v = 0.f;
 #pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                float* r = rb + ((size_t)warp * NT + n) * 128;
-                *reinterpret_cast<float2*>(r + g * 8 + 2 * t) = make_float2(acc[n][0], acc[n][1]);
-                *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) = make_float2(acc[n][2], acc[n][3]);
+                        for (int w = 0; w < NWARPS; ++w) v += V == 4 ? rb[w * NACC * 128] + rb[w * NACC * 128 + 4] : rb[w * NACC * 128];
+                        float* dst = acc_s + (size_t)((si >> 1) * 16 + r16) * MP + m;
+                        *dst = ph == 0 ? v : *dst + v;
+                    }
+                }
+                KG_PROBE(14);
+                buf ^= 1;
             }
         }
-        __syncthreads();
-        if (!rs_ready) {      // 1/rms per row, summed over warps in a fixed order (same value in every thread)
-            rs_ready = true;
+        // ---- epilogue of this superchunk
+        if (sc0 == pl.u0) {
+            // 1/rms per activation row: the four lanes sharing g hold the partial sums of row xrow (+ 8)
+#pragma unroll
+            for (int n = 0; n < NACC; ++n) {
+                float s = ssq[n];
+                s += __shfl_xor_sync(0xffffffffu, s, 1);
+                s += __shfl_xor_sync(0xffffffffu, s, 2);
+                if (t == 0 && (V != 4 || g < 4)) ssw[warp * M_MAX + xrow + 8 * n] = s;
+            }
+        }
+        cta_sync();
+        if (sc0 == pl.u0) {
             if (tid < M_MAX) {
                 float r = 1.0f;
                 if (a.gain && tid < M) {
@@ -372,80 +607,73 @@ __device__ void lin_mma(const LinArgs& a, Ctx& c) {
                 }
                 rs[tid] = r;
             }
-            __syncthreads();
+            cta_sync();
         }
-        // value of (tile-local row r16, activation row m) summed over the k-slices in order
-        auto reduced = [&](int tile, int r16, int m) -> float {
-            const float* r = rb + ((size_t)(tile * n_ks) * NT + (m >> 3)) * 128 + r16 * 8 + (m & 7);
-            float v = 0.f;
-            for (int ks = 0; ks < n_ks; ++ks) v += r[(size_t)ks * NT * 128];
-            return v;
-        };
         if (a.epi == EPI_SWIGLU) {
-            const int nf = min(nt * 8, nr - t0 * 8);
-            for (int idx = tid; idx < nf * M; idx += NTHREADS) {
-                const int fl = idx % nf, m = idx / nf;
-                const float vg = reduced(fl >> 3, fl & 7, m) * rs[m];
-                const float vu = reduced(fl >> 3, (fl & 7) + 8, m) * rs[m];
-                a.out[(size_t)m * a.ldo + r0 + t0 * 8 + fl] = silu_f(vg) * vu;
+            for (int idx = tid; idx < nu * M; idx += NTHREADS) {
+                const int fl_ = idx % nu, m = idx / nu;
+                const int srow = (fl_ >> 3) * 16 + (fl_ & 7);
+                const float vg = acc_s[(size_t)srow * MP + m] * rs[m];
+                const float vu = acc_s[(size_t)(srow + 8) * MP + m] * rs[m];
+                a.out[(size_t)m * a.ldo + sc0 + fl_] = silu_f(vg) * vu;
             }
         } else if (a.epi == EPI_HEAD) {
-            const int nrow = min(nt * 16, nr - t0 * 16);
-            if (warp < M) {
-                const int m = warp;
-                float zl[2]; int il[2];
-                float zm = -INFINITY; int im = 0x7fffffff;
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    const int r = lane + 32 * q;
-                    zl[q] = -INFINITY; il[q] = 0x7fffffff;
-                    if (r < nrow) {
-                        zl[q] = reduced(r >> 4, r & 15, m) * rs[m] * a.scale;
-                        il[q] = (int)(r0 + t0 * 16 + r);
-                        if (a.logits_dbg) a.logits_dbg[(size_t)m * a.ld_dbg + il[q]] = zl[q];
-                        if (arg_better(zl[q], il[q], zm, im)) { zm = zl[q]; im = il[q]; }
+            for (int q = 0; q < 2; ++q) {
+                const int m = warp + q * NWARPS;
+                if (m < M) {
+                    const float f = rs[m] * a.scale;
+                    float zm = -INFINITY; int im = 0x7fffffff;
+                    for (int r = lane; r < nu; r += 32) {
+                        const float z = acc_s[(size_t)r * MP + m] * f;
+                        if (a.logits_dbg) a.logits_dbg[(size_t)m * a.ld_dbg + sc0 + r] = z;
+                        if (arg_better(z, sc0 + r, zm, im)) { zm = z; im = sc0 + r; }
                     }
-                }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    float z2 = __shfl_xor_sync(0xffffffffu, zm, o);
-                    int i2 = __shfl_xor_sync(0xffffffffu, im, o);
-                    if (arg_better(z2, i2, zm, im)) { zm = z2; im = i2; }
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const float z2 = __shfl_xor_sync(0xffffffffu, zm, o);
+                        const int i2 = __shfl_xor_sync(0xffffffffu, im, o);
+                        if (arg_better(z2, i2, zm, im)) { zm = z2; im = i2; }
+                    }
+                    float e = 0.f;
+                    for (int r = lane; r < nu; r += 32) e += expf(acc_s[(size_t)r * MP + m] * f - zm);
+                    e = warp_sum(e);
+                    if (nu > 0) head_merge(hs[q], zm, e, im);
                 }
-                float e = 0.f;
-#pragma unroll
-                for (int q = 0; q < 2; ++q) if (lane + 32 * q < nrow) e += expf(zl[q] - zm);
-                e = warp_sum(e);
-                head_merge(hs, zm, e, im);
             }
         } else {
-            const int nrow = min(nt * 16, nr - t0 * 16);
-            for (int idx = tid; idx < nrow * M; idx += NTHREADS) {
-                const int r = idx % nrow, m = idx / nrow;
-                float v = reduced(r >> 4, r & 15, m) * rs[m];
-                const size_t row = (size_t)(r0 + t0 * 16 + r);
+            for (int idx = tid; idx < nu * M; idx += NTHREADS) {
+                const int r = idx % nu, m = idx / nu;
+                float v = acc_s[(size_t)r * MP + m] * rs[m];
+                const size_t row = (size_t)(sc0 + r);
                 if (a.epi == EPI_RESID) v += ldcg_f(a.resid + (size_t)m * a.ldr + row);
                 a.out[(size_t)m * a.ldo + row] = v;
             }
         }
-        buf ^= 1;
+        cta_sync();                                  // acc_s and the staged rows are rewritten by the next superchunk / operator
+        KG_PROBE(15);
     }
-    if (a.epi == EPI_HEAD && warp < M && lane == 0)
-        a.head_part[(size_t)c.cta * M_MAX + warp] = make_float4(hs.zmax, hs.sum, __int_as_float(hs.arg), 0.f);
-    __syncthreads();
+    if (a.epi == EPI_HEAD && lane == 0) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int m = warp + q * NWARPS;
+            if (m < M) a.head_part[(size_t)c.cta * M_MAX + m] = make_float4(hs[q].zmax, hs[q].sum, __int_as_float(hs[q].arg), 0.f);
+        }
+    }
 }
 
-// Plain path for any storage type (used for fp32 models and as a cross-check of the tensor-core
+// Plain path for any storage type (fp32 models, odd shapes, and a cross-check of the tensor-core
 // path): activations staged in shared memory as fp32, one output row per warp at a time.
 template <typename WT>
-__device__ void lin_simple(const LinArgs& a, Ctx& c) {
+__device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M, K = a.K;
     const WT* W = reinterpret_cast<const WT*>(a.W);
     const WT* W2 = reinterpret_cast<const WT*>(a.W2);
     const bool dual = W2 != nullptr;
-    float* xs = reinterpret_cast<float*>(c.smem);                        // [M][K]
-    float* rs = reinterpret_cast<float*>(c.smem + XS_BUDGET);            // [M_MAX]
+    char* work = c.smem + WORK_OFF;
+    float* xs = reinterpret_cast<float*>(work);                          // [M][K]
+    float* rs = reinterpret_cast<float*>(work + SIMPLE_XS_BYTES);        // [M_MAX]
     float* wst = rs + M_MAX;                                             // [NWARPS][M_MAX][3] head stats
 
     for (int m = warp; m < M; m += NWARPS) {
@@ -458,7 +686,7 @@ __device__ void lin_simple(const LinArgs& a, Ctx& c) {
         ss = warp_sum(ss);
         if (lane == 0) rs[m] = a.gain ? rsqrtf(ss / (float)K + a.eps) : 1.0f;
     }
-    __syncthreads();
+    cta_sync();
 
     HeadStat hs; hs.zmax = 0.f; hs.sum = 0.f; hs.arg = 0;               // lane m tracks row m
     for (long long row = (long long)c.cta * NWARPS + warp; row < a.N; row += (long long)c.nctas * NWARPS) {
@@ -502,7 +730,7 @@ __device__ void lin_simple(const LinArgs& a, Ctx& c) {
             wst[(warp * M_MAX + lane) * 3 + 1] = hs.sum;
             wst[(warp * M_MAX + lane) * 3 + 2] = __int_as_float(hs.arg);
         }
-        __syncthreads();
+        cta_sync();
         if (tid < M) {
             HeadStat tot; tot.zmax = 0.f; tot.sum = 0.f; tot.arg = 0;
             for (int w = 0; w < NWARPS; ++w)
@@ -511,20 +739,29 @@ __device__ void lin_simple(const LinArgs& a, Ctx& c) {
             a.head_part[(size_t)c.cta * M_MAX + tid] = make_float4(tot.zmax, tot.sum, __int_as_float(tot.arg), 0.f);
         }
     }
-    __syncthreads();
+    cta_sync();
 }
 
-template <typename WT> struct LinDispatch;
-template <> struct LinDispatch<float> {
-    static __device__ __forceinline__ void run(const LinArgs& a, Ctx& c, bool) { lin_simple<float>(a, c); }
-};
-template <> struct LinDispatch<__nv_bfloat16> {
-    static __device__ __forceinline__ void run(const LinArgs& a, Ctx& c, bool force_simple) {
-        if (force_simple || (a.K & 31) != 0) lin_simple<__nv_bfloat16>(a, c);
-        else if (a.M <= 8) lin_mma<1>(a, c);
-        else lin_mma<2>(a, c);
+// Which path an operator takes; the producer and the consumers must agree.
+template <typename WT> __device__ __forceinline__ bool lin_streams(const LinArgs& a, bool force_simple);
+template <> __device__ __forceinline__ bool lin_streams<float>(const LinArgs&, bool) { return false; }
+template <> __device__ __forceinline__ bool lin_streams<__nv_bfloat16>(const LinArgs& a, bool force_simple) {
+    return !force_simple && (a.K & 15) == 0;
+}
+
+// One linear operator, called by every thread of the CTA.  Consumers return after their part;
+// whether the grid must stop is learnt at the next grid barrier.  The producer returns false when
+// one of its waits gave up.
+template <typename WT>
+__device__ __forceinline__ bool linear_op(const LinArgs& a, Ctx& c, bool force_simple) {
+    if (lin_streams<WT>(a, force_simple)) {
+        if (c.producer) return lin_produce(a, c);
+        if (a.M <= 4) lin_consume<4>(a, c); else if (a.M <= 8) lin_consume<8>(a, c); else lin_consume<16>(a, c);
+        return true;
     }
-};
+    if (!c.producer) lin_simple<WT>(a, c);
+    return true;
+}
 
 // Merge the per-CTA head partials of row m (identical result in every CTA: fixed order).
 __device__ __forceinline__ void head_final(const float4* part, int nctas, int m, int& tok, float& p) {
@@ -545,12 +782,12 @@ struct AttArgs {
     float* out;            // [M][d]
 };
 
-// One work item = (head, KV split).  Keys come from the paged cache; the rows of this pass are
-// rotated (RoPE), rounded to the cache's storage type and appended to the cache by the item whose
-// key range contains them, then read back like any other key.  Every split writes a partial
-// (max, sum, o); the last split of a head to arrive merges them in split order.
+// Consumer threads only.  One work item = (head, KV split).  Keys come from the paged cache; the
+// rows of this pass are rotated (RoPE), rounded to the cache's storage type and appended to the
+// cache by the item whose key range contains them, then read back like any other key.  Every split
+// writes a partial (max, sum, o); the last split of a head to arrive merges them in split order.
 template <typename WT>
-__device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
+__device__ __noinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int H = D.dm.H, hd = D.dm.hd, d = D.dm.d, ps = D.dm.page_size;
     const int M = a.M, pos0 = a.pos0;
@@ -562,23 +799,23 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
     WT* kc = reinterpret_cast<WT*>(a.kc);
     WT* vc = reinterpret_cast<WT*>(a.vc);
 
-    float* qs = reinterpret_cast<float*>(c.smem);                  // [M_MAX][HD_MAX]
+    float* qs = reinterpret_cast<float*>(c.smem + WORK_OFF);       // [M_MAX][HD_MAX]
     float* Ks = qs + M_MAX * HD_MAX;                               // [ATT_TK][hd+4]
     float* Vs = Ks + ATT_TK * (HD_MAX + 4);                        // [ATT_TK][hd]
     float* Ss = Vs + ATT_TK * HD_MAX;                              // [M_MAX][ATT_TK]
     float* mrun = Ss + M_MAX * ATT_TK;                             // [M_MAX] running max
     float* lrun = mrun + M_MAX;                                    // [M_MAX] running sum
     float* corr = lrun + M_MAX;                                    // [M_MAX]
-    __shared__ int s_last;
     const int kstr = hd + 4;
     const int rgs = NTHREADS / hd;                                 // row groups in the PV phase
     const int e_pv = tid % hd, rg_pv = tid / hd;
-    constexpr int PV_R = 4;                                        // rows per thread in PV (rgs >= 4)
+    constexpr int PV_R = 8;                                        // rows per thread in PV (rgs >= 2)
+    constexpr int SC_G = NTHREADS / ATT_TK;                        // row groups in the score phase
 
     for (int item = c.cta; item < H * S; item += c.nctas) {
         const int hh = item / S, s = item % S;
         const int kb = s * chunk, ke = min(T, kb + chunk);
-        __syncthreads();
+        cta_sync();
         // q rows: RoPE, pre-scaled by 1/sqrt(hd)
         for (int idx = tid; idx < M * half; idx += NTHREADS) {
             const int i = idx / half, e = idx % half;
@@ -607,7 +844,7 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
         float o[PV_R];
 #pragma unroll
         for (int r = 0; r < PV_R; ++r) o[r] = 0.f;
-        __syncthreads();
+        cta_sync();
 
         for (int tb = kb; tb < ke; tb += ATT_TK) {
             const int nk = min(ATT_TK, ke - tb);
@@ -620,34 +857,28 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
                 *reinterpret_cast<float4*>(Ks + j * kstr + e4) = kv;
                 *reinterpret_cast<float4*>(Vs + j * hd + e4) = vv;
             }
-            __syncthreads();
-            // scores: thread (key j, row group) -> rows i = rgq, rgq + 8
+            cta_sync();
+            // scores: thread (key j, row group rgq) -> rows i = rgq, rgq + SC_G, ...
             {
-                const int j = tid % ATT_TK, rgq = tid / ATT_TK;          // 8 row groups
-                float s0 = 0.f, s1 = 0.f;
-                const bool r0v = rgq < M, r1v = rgq + 8 < M;
-                if (j < nk && r0v) {
-                    const float* kr = Ks + j * kstr;
-                    const float* q0 = qs + rgq * HD_MAX;
-                    const float* q1 = qs + (rgq + 8) * HD_MAX;
-                    for (int e4 = 0; e4 < hd; e4 += 4) {
-                        const float4 kv = *reinterpret_cast<const float4*>(kr + e4);
-                        const float4 a0 = *reinterpret_cast<const float4*>(q0 + e4);
-                        s0 = fmaf(kv.x, a0.x, fmaf(kv.y, a0.y, fmaf(kv.z, a0.z, fmaf(kv.w, a0.w, s0))));
-                        if (r1v) {
-                            const float4 a1 = *reinterpret_cast<const float4*>(q1 + e4);
-                            s1 = fmaf(kv.x, a1.x, fmaf(kv.y, a1.y, fmaf(kv.z, a1.z, fmaf(kv.w, a1.w, s1))));
+                const int j = tid % ATT_TK, rgq = tid / ATT_TK;
+                const int pos = tb + j;
+                for (int i = rgq; i < M; i += SC_G) {
+                    float s0 = 0.f;
+                    if (j < nk) {
+                        const float* kr = Ks + j * kstr;
+                        const float* q0 = qs + i * HD_MAX;
+                        for (int e4 = 0; e4 < hd; e4 += 4) {
+                            const float4 kv = *reinterpret_cast<const float4*>(kr + e4);
+                            const float4 a0 = *reinterpret_cast<const float4*>(q0 + e4);
+                            s0 = fmaf(kv.x, a0.x, fmaf(kv.y, a0.y, fmaf(kv.z, a0.z, fmaf(kv.w, a0.w, s0))));
                         }
                     }
+                    Ss[i * ATT_TK + j] = (j < nk && pos <= pos0 + i) ? s0 : -INFINITY;
                 }
-                const int pos = tb + j;
-                if (r0v) Ss[rgq * ATT_TK + j] = (j < nk && pos <= pos0 + rgq) ? s0 : -INFINITY;
-                if (r1v) Ss[(rgq + 8) * ATT_TK + j] = (j < nk && pos <= pos0 + rgq + 8) ? s1 : -INFINITY;
             }
-            __syncthreads();
-            // online softmax bookkeeping: warp i owns row i
-            if (warp < M) {
-                const int i = warp;
+            cta_sync();
+            // online softmax bookkeeping: warp i owns rows i, i + NWARPS
+            for (int i = warp; i < M; i += NWARPS) {
                 const float v0 = Ss[i * ATT_TK + lane], v1 = Ss[i * ATT_TK + lane + 32];
                 const float mo = mrun[i];
                 const float mn = fmaxf(mo, warp_max(fmaxf(v0, v1)));
@@ -660,7 +891,7 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
                 const float ps_ = warp_sum(p0 + p1);
                 if (lane == 0) { lrun[i] = lrun[i] * cf + ps_; mrun[i] = mn; corr[i] = cf; }
             }
-            __syncthreads();
+            cta_sync();
             // o += P V : thread (element e, row group) -> rows i = rg_pv + rgs * r
             if (rg_pv < rgs) {
 #pragma unroll
@@ -674,7 +905,7 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
                     }
                 }
             }
-            __syncthreads();
+            cta_sync();
         }
         // partials
         if (rg_pv < rgs) {
@@ -689,14 +920,15 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
             D.att_ml[(((size_t)tid * H + hh) * S_CAP + s) * 2 + 1] = lrun[tid];
         }
         __threadfence();
-        __syncthreads();
+        cta_sync();
         if (tid == 0) {
             const unsigned prev = atomicAdd(D.att_cnt + hh, 1u);
-            s_last = (prev == (unsigned)(S - 1));
-            if (s_last) { D.att_cnt[hh] = 0u; __threadfence(); }
+            const int last = (prev == (unsigned)(S - 1));
+            c.ctl->att_last = last;
+            if (last) { D.att_cnt[hh] = 0u; __threadfence(); }
         }
-        __syncthreads();
-        if (s_last) {
+        cta_sync();
+        if (*(volatile int*)&c.ctl->att_last) {
             for (int idx = tid; idx < M * hd; idx += NTHREADS) {
                 const int i = idx / hd, e = idx % hd;
                 const float* ml = D.att_ml + ((size_t)i * H + hh) * S_CAP * 2;
@@ -714,13 +946,12 @@ __device__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
             }
         }
     }
-    __syncthreads();
+    cta_sync();
 }
 
-__host__ __device__ inline size_t smem_bytes_needed() {
-    size_t lin = (size_t)XS_BUDGET + (2 * NWARPS * 2 * 128 + NWARPS * M_MAX + M_MAX + NWARPS * M_MAX * 3 + 64) * sizeof(float);
-    size_t att = (size_t)(M_MAX * HD_MAX + ATT_TK * (HD_MAX + 4) + ATT_TK * HD_MAX + M_MAX * ATT_TK + 3 * M_MAX) * sizeof(float);
-    return lin > att ? lin : att;
-}
+static_assert((M_MAX * HD_MAX + ATT_TK * (HD_MAX + 4) + ATT_TK * HD_MAX + M_MAX * ATT_TK + 3 * M_MAX) * 4 <= WORK_BYTES,
+              "attention tiles do not fit in the work area");
+static_assert(9 * (LinGeom<8>::PLEN * 4 + 32) + (2 * NWARPS * 128 + SC_ROWS * MP + NWARPS * M_MAX + M_MAX) * 4 <= WORK_BYTES, "linear work area too large (M <= 8)");
+static_assert(17 * (LinGeom<16>::PLEN * 4 + 32) + (2 * NWARPS * 128 + SC_ROWS * MP + NWARPS * M_MAX + M_MAX) * 4 <= WORK_BYTES, "linear work area too large (M <= 16)");
 
 }  // namespace kg

@@ -2,6 +2,12 @@
 // method - prefill chunks, the draft loop with its on-device exit test, the verify pass, the
 // prefix accept / rollback, or many rounds back to back - with grid barriers between dependent
 // operators and no host involvement.
+//
+// Every thread of every CTA walks the same operator sequence and holds the same copy of the
+// sequence state.  The consumer warps do the arithmetic and take part in the grid barriers; the
+// producer warp only issues the weight copies of each linear operator, so it runs ahead of the
+// consumers (through barriers and attention) until the next decision that depends on a result
+// (a drafted token, its confidence, the accepted prefix), which it receives through shared memory.
 #pragma once
 
 #include "kg_device.cuh"
@@ -17,7 +23,8 @@ struct Program {
     int force_simple;   // 1: route bf16 linears through the plain path (cross-check)
 };
 
-#define KG_SYNC(where) do { if (!grid_sync(c, (where))) return false; } while (0)
+#define KG_SYNC(where) do { if (!sync(where)) return false; } while (0)
+#define KG_LIN(args) do { if (!linear(args)) return false; } while (0)
 
 template <typename WT>
 struct Engine {
@@ -27,7 +34,10 @@ struct Engine {
 
     __device__ Engine(const Dev& d, Ctx& cx, const Program& p) : D(d), c(cx), pg(p) {}
 
-    __device__ __forceinline__ void linear(const LinArgs& a) { LinDispatch<WT>::run(a, c, pg.force_simple != 0); }
+    // ---- leaf operations: what a thread does depends on its role -------------------------------
+    __device__ __forceinline__ bool linear(const LinArgs& a) { return linear_op<WT>(a, c, pg.force_simple != 0); }
+    __device__ __forceinline__ bool sync(int where) { return c.producer ? true : grid_sync(c, where); }
+    __device__ __forceinline__ void attention(const AttArgs& at) { if (!c.producer) attention_op<WT>(D, at, c); }
 
     __device__ size_t cache_layer_stride() const {
         return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
@@ -35,6 +45,7 @@ struct Engine {
 
     // h[i] = E[token_i]
     __device__ void embed_rows(const int* toks_global, int tok_single, int M, float* out) {
+        if (c.producer) return;
         const int d = D.dm.d;
         const WT* E = reinterpret_cast<const WT*>(D.embed);
         for (int idx = c.cta * NTHREADS + threadIdx.x; idx < M * d; idx += c.nctas * NTHREADS) {
@@ -54,28 +65,28 @@ struct Engine {
         // q, k, v
         a.W = lw.wqkv; a.W2 = nullptr; a.N = 3 * dm.d; a.K = dm.d;
         a.x = xin; a.ldx = dm.d; a.gain = lw.g1; a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(10);
         AttArgs at;
         at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
         at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)li * cache_layer_stride();
         at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)li * cache_layer_stride();
         at.out = D.attn;
-        attention_op<WT>(D, at, c);
+        attention(at);
         KG_SYNC(11);
         // output projection + residual -> h
         a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
         a.epi = EPI_RESID; a.resid = xin; a.ldr = dm.d; a.out = D.h; a.ldo = dm.d;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(12);
         // SwiGLU
         a.W = lw.wgate; a.W2 = lw.wup; a.N = dm.F; a.K = dm.d; a.x = D.h; a.ldx = dm.d; a.gain = lw.g2;
         a.epi = EPI_SWIGLU; a.out = D.act; a.ldo = dm.F;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(13);
         a.W = lw.wdown; a.W2 = nullptr; a.N = dm.d; a.K = dm.F; a.x = D.act; a.ldx = dm.F; a.gain = nullptr;
         a.epi = EPI_RESID; a.resid = D.h; a.ldr = dm.d; a.out = out; a.ldo = dm.d;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(14);
         return true;
     }
@@ -89,25 +100,26 @@ struct Engine {
         a.M = M; a.eps = dm.eps;
         a.W = lw.wqkv; a.N = 3 * dm.d; a.K = dm.d; a.x = f; a.ldx = dm.d; a.gain = lw.g1;
         a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(20);
         AttArgs at;
         at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
         at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)dm.L * cache_layer_stride();
         at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)dm.L * cache_layer_stride();
         at.out = D.attn;
-        attention_op<WT>(D, at, c);
+        attention(at);
         KG_SYNC(21);
         if (!want_out) return true;
         a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
         a.epi = EPI_RESID; a.resid = f; a.ldr = dm.d; a.out = D.abuf; a.ldo = dm.d;
-        linear(a);
+        KG_LIN(a);
         KG_SYNC(22);
         return true;
     }
 
-    // Shared LM head on rows x[M] (norm gain `gain`), then the merged (token, p) per row, the same
-    // values in every thread of every CTA.
+    // Shared LM head on rows x[M] (norm gain `gain`), then the merged (token, p) per row: the same
+    // values in every thread of every CTA, the producer warp included (it receives them through
+    // shared memory and an mbarrier, which also holds it back until the result exists).
     __device__ bool run_head(const float* x, int M, const float* gain, float* dbg, int* toks, float* ps) {
         const Dims& dm = D.dm;
         LinArgs a{};
@@ -115,18 +127,25 @@ struct Engine {
         a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = x; a.ldx = dm.d; a.gain = gain;
         a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
         a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
-        linear(a);
-        KG_SYNC(30);
-        __shared__ int s_tok[M_MAX];
-        __shared__ float s_p[M_MAX];
-        if (threadIdx.x < M) {
-            int tk; float p;
-            head_final(D.head_part, c.nctas, threadIdx.x, tk, p);
-            s_tok[threadIdx.x] = tk; s_p[threadIdx.x] = p;
+        if (!linear(a)) return false;
+        if (c.producer) {
+            // held back here until the consumers have the result
+            int ok = 1;
+            if ((threadIdx.x & 31) == 0) ok = mbar_wait(c, &c.ctl->mail, c.mail_phase, 42) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            c.mail_phase ^= 1u;
+            if (!ok) return false;
+        } else {
+            if (!grid_sync(c, 30)) return false;
+            if (threadIdx.x < M) {
+                int tk; float p;
+                head_final(D.head_part, c.nctas, threadIdx.x, tk, p);
+                c.ctl->head_tok[threadIdx.x] = tk; c.ctl->head_p[threadIdx.x] = p;
+            }
+            cta_sync();
+            if (threadIdx.x == 0) mbar_arrive(&c.ctl->mail);
         }
-        __syncthreads();
-        for (int i = 0; i < M; ++i) { toks[i] = s_tok[i]; ps[i] = s_p[i]; }
-        __syncthreads();
+        for (int i = 0; i < M; ++i) { toks[i] = c.ctl->head_tok[i]; ps[i] = c.ctl->head_p[i]; }
         return true;
     }
 
@@ -199,7 +218,7 @@ struct Engine {
         while (k < n_d && dtok[k] == t[k]) ++k;
         const int newP = P + k + 1;
         if (len_A > newP) len_A = newP;
-        if (len_A < newP) {
+        if (len_A < newP && !c.producer) {
             // the adapter has not seen f[k] (k == n_d): keep it as the feature of position newP-1
             const float* src = D.feat + (size_t)(1 + k) * dm.d;
             for (int e = c.cta * NTHREADS + threadIdx.x; e < dm.d; e += c.nctas * NTHREADS) D.feat[e] = __ldcg(src + e);
@@ -224,6 +243,7 @@ struct Engine {
         const Dims& dm = D.dm;
         const int n = pg.n;
         int tk[M_MAX]; float pp[M_MAX];
+        tk[0] = 0;
         for (int c0 = 0; c0 < n; c0 += M_MAX) {
             const int M = min(M_MAX, n - c0);
             embed_rows(D.prompt + c0, 0, M, D.h);
@@ -259,28 +279,34 @@ struct Engine {
         return true;
     }
 
-    __device__ void run() {
-        load_state();
+    __device__ bool run_program() {
         switch (pg.kind) {
-            case PROG_PREFILL: prefill(); break;
-            case PROG_DRAFT: draft_phase(); break;
-            case PROG_VERIFY: verify_phase(); break;
-            case PROG_AR: ar_decode(); break;
+            case PROG_PREFILL: return prefill();
+            case PROG_DRAFT: return draft_phase();
+            case PROG_VERIFY: return verify_phase();
+            case PROG_AR: return ar_decode();
             case PROG_DECODE:
                 while (total < pg.n) {
-                    if (!draft_phase()) return;
-                    if (!verify_phase()) return;
+                    if (!draft_phase()) return false;
+                    if (!verify_phase()) return false;
                 }
-                break;
+                return true;
         }
+        return true;
+    }
+
+    __device__ void run() {
+        load_state();
+        const bool ok = run_program();
+        if (!ok && c.producer) ring_drain(c);
     }
 };
 
 template <typename WT>
-__global__ void __launch_bounds__(NTHREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
     extern __shared__ __align__(128) char smem[];
     Ctx c;
-    c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = D.st; c.bar = D.bar; c.smem = smem; c.grid = true;
+    ctx_init(c, smem, D.st, D.bar, true);
     Engine<WT> eng(D, c, pg);
     eng.run();
 }
