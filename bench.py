@@ -228,6 +228,10 @@ def run_kangaroo(args):
     shape = ki.get_config(args.workload)
     if args.n_gen:
         shape = shape.with_(n_gen=args.n_gen)
+    if args.n_prompt:
+        shape = shape.with_(n_prompt=args.n_prompt)
+    if args.layers:
+        shape = shape.with_(n_layers=args.layers, name=f"{shape.name}-{args.layers}layers")
     mode = binding.STOP_DROP if args.stop == "drop" else binding.STOP_KEEP
     model = binding.KangarooModel(shape, device=f"cuda:{local_rank}")
     prompt_np = ki.make_prompt(shape)
@@ -342,6 +346,8 @@ def main():
     ap.add_argument("--workload", default="7b", choices=["tiny", "7b", "13b", "33b"])
     ap.add_argument("--stop", default="keep", choices=["keep", "drop"])
     ap.add_argument("--n-gen", type=int, default=0, help="override the number of generated tokens (debugging)")
+    ap.add_argument("--n-prompt", type=int, default=0, help="override the prompt length (profiling on a small case)")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling on a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kangaroo" else args.warmup
