@@ -34,7 +34,8 @@ typedef enum {
     KG_E_NOMEM = -3,     /* arena too small */
     KG_E_SEQ_FULL = -4,  /* the sequence would exceed max_seq */
     KG_E_CUDA = -5,      /* a CUDA runtime call failed */
-    KG_E_TIMEOUT = -6    /* a bounded device-side wait expired; the model must be re-initialised */
+    KG_E_TIMEOUT = -6,   /* a bounded device-side wait expired; the model must be re-initialised */
+    KG_E_LIMIT = -7      /* a size exceeds what a fixed-capacity entry point (kg_op_lm_head_noalloc) can hold */
 } kg_status;
 
 enum { KG_F32 = 0, KG_BF16 = 1 };            /* storage type of weights and KV cache */
@@ -187,6 +188,23 @@ int kg_op_linear(int32_t dtype, const void* W_dev, const void* W2_dev, int32_t N
 int kg_op_lm_head(int32_t dtype, const void* W_head_dev, int32_t V, int32_t K, const float* x_dev, int32_t M,
                   const float* gain_dev, float eps, float logit_scale,
                   int32_t* tok_dev, float* p_dev, float* logits_dev, void* scratch_dev, void* cuda_stream);
+
+/* kg_op_lm_head without any caller scratch and without any allocation (the paper has no counterpart: this is
+ * a deployment convenience).  It is for callers that cannot obtain device memory at the time of the call -
+ * code running while a memory pool is frozen or exhausted, inside a plugin whose host forbids cudaMalloc, or
+ * in an error path that must still produce a token.  The per-CTA partial results that kg_op_lm_head keeps in
+ * `scratch_dev` live here in a 64 KB array that is part of the library image, so every GPU that loads the
+ * library holds those 64 KB until the process exits.
+ * Limits: M <= KG_M_MAX rows and a device with at most 256 SMs (one partial per SM and row); anything larger
+ * returns KG_E_LIMIT.  V and K are not limited: W, x and the outputs remain caller memory.
+ * The first call on each device looks up the array's device address (no allocation); make that first call
+ * outside any stream capture.  All calls share the one array: two calls whose kernels overlap on the GPU
+ * (different streams, no ordering between them) race on it and give wrong results; calls ordered on one
+ * stream are safe, and nothing in the array has to be cleared between calls because every partial is
+ * rewritten before it is read. */
+int kg_op_lm_head_noalloc(int32_t dtype, const void* W_head_dev, int32_t V, int32_t K, const float* x_dev, int32_t M,
+                          const float* gain_dev, float eps, float logit_scale,
+                          int32_t* tok_dev, float* p_dev, float* logits_dev, void* cuda_stream);
 
 /* Causal attention of M new rows at positions pos0.. over a paged KV cache (RoPE fused): takes the
  * raw q,k,v rows qkv[M, 3d], rotates q and k, appends k and v to the cache pages, and returns

@@ -17,13 +17,13 @@ KG_GAMMA_MAX = KG_M_MAX - 1
 KG_F32, KG_BF16 = 0, 1
 STOP_KEEP, STOP_DROP = 0, 1
 
-KG_OK, KG_E_ARG, KG_E_STATE, KG_E_NOMEM, KG_E_SEQ_FULL, KG_E_CUDA, KG_E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+KG_OK, KG_E_ARG, KG_E_STATE, KG_E_NOMEM, KG_E_SEQ_FULL, KG_E_CUDA, KG_E_TIMEOUT, KG_E_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7
 
 EXPORTS = [
     "kg_workspace_bytes", "kg_init_model", "kg_free_model", "kg_reset", "kg_prefill", "kg_prefill_device",
     "kg_draft", "kg_verify", "kg_decode", "kg_decode_ar", "kg_generate", "kg_read_tokens", "kg_read_S", "kg_read_round_log",
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
-    "kg_op_lm_head", "kg_op_attention", "kg_strerror",
+    "kg_op_lm_head", "kg_op_lm_head_noalloc", "kg_op_attention", "kg_strerror",
 ]
 
 
@@ -108,6 +108,7 @@ def load():
     lib.kg_op_scratch_bytes.argtypes = []
     lib.kg_op_linear.argtypes = [i32, vp, vp, i32, i32, vp, i32, vp, f32, vp, i32, vp, vp, vp]
     lib.kg_op_lm_head.argtypes = [i32, vp, i32, i32, vp, i32, vp, f32, f32, vp, vp, vp, vp, vp]
+    lib.kg_op_lm_head_noalloc.argtypes = [i32, vp, i32, i32, vp, i32, vp, f32, f32, vp, vp, vp, vp]
     lib.kg_op_attention.argtypes = [i32, vp, i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, vp, vp]
     lib.kg_strerror.restype = C.c_char_p
     lib.kg_strerror.argtypes = [C.c_int]
@@ -315,6 +316,18 @@ def op_lm_head(W, x, gain, eps, logit_scale, want_logits=True, scratch=None):
     _check(lib.kg_op_lm_head(dt, W.data_ptr(), V, K, x.data_ptr(), M, _ptr(gain), eps, logit_scale,
                              tok.data_ptr(), p.data_ptr(), _ptr(logits), scratch.data_ptr(), _stream(torch)), "kg_op_lm_head")
     return tok, p, logits
+
+
+def op_lm_head_noalloc(W, x, gain, eps, logit_scale, tok, p, logits=None):
+    """kg_op_lm_head_noalloc on caller-made tensors: tok (int32 [M]), p (float32 [M]) and optionally logits
+    (float32 [M, V]) must exist already, so the call itself allocates nothing on the device."""
+    import torch
+    lib = load()
+    V, K = W.shape
+    M = x.shape[0]
+    dt = KG_BF16 if W.dtype == torch.bfloat16 else KG_F32
+    _check(lib.kg_op_lm_head_noalloc(dt, W.data_ptr(), V, K, x.data_ptr(), M, _ptr(gain), eps, logit_scale,
+                                     tok.data_ptr(), p.data_ptr(), _ptr(logits), _stream(torch)), "kg_op_lm_head_noalloc")
 
 
 def op_attention(qkv, pos0, n_heads, head_dim, rope_theta, kcache, vcache, page_table, page_size, scratch=None):

@@ -190,6 +190,7 @@ extern "C" const char* kg_strerror(int s) {
         case KG_E_SEQ_FULL: return "sequence would exceed max_seq";
         case KG_E_CUDA: return "CUDA runtime error";
         case KG_E_TIMEOUT: return "device-side wait timed out";
+        case KG_E_LIMIT: return "size beyond the capacity of the library's static scratch";
         default: return "unknown status";
     }
 }
@@ -772,6 +773,51 @@ extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K,
     a.epi = EPI_HEAD; a.scale = logit_scale; a.head_part = (float4*)((char*)scratch + sc.off_hp);
     a.logits_dbg = logits; a.ld_dbg = V;
     int r = op_linear_common(dtype, a, (cudaStream_t)stream);
+    if (r != KG_OK) return r;
+    op_head_final_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(a.head_part, sm_count(), M, tok, p);
+    CK(cudaGetLastError());
+    return KG_OK;
+}
+
+// ------------------------------------------------------------------------------------ no-allocation variant
+// The LM-head operator keeps one partial (max, sum, arg max) per CTA and row in scratch memory.  Here that
+// scratch is a fixed array inside the library image instead of caller memory.
+namespace {
+constexpr int NOALLOC_MAX_CTAS = 256;                        // CTAs (one per SM) the static scratch has room for
+constexpr int NOALLOC_MAX_DEVICES = 64;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(float4) * NOALLOC_MAX_CTAS * KG_M_MAX];   // 64 KB
+void* g_noalloc_addr[NOALLOC_MAX_DEVICES] = {nullptr};
+
+// Device address of the static scratch on the current device.  In host code the array's name is only a
+// handle for the runtime, never a pointer a kernel may use; the address comes from cudaGetSymbolAddress.
+int noalloc_scratch(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KG_E_CUDA;
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return KG_E_LIMIT;
+    if (!g_noalloc_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return KG_E_CUDA;
+        g_noalloc_addr[dev] = p;
+    }
+    *out = g_noalloc_addr[dev];
+    return KG_OK;
+}
+}  // namespace
+
+extern "C" int kg_op_lm_head_noalloc(int32_t dtype, const void* W, int32_t V, int32_t K, const float* x, int32_t M,
+                                     const float* gain, float eps, float logit_scale,
+                                     int32_t* tok, float* p, float* logits, void* stream) {
+    if (!W || !x || !tok || !p) return KG_E_ARG;
+    if (M > KG_M_MAX || sm_count() > NOALLOC_MAX_CTAS) return KG_E_LIMIT;
+    void* scratch = nullptr;
+    int r = noalloc_scratch(&scratch);
+    if (r != KG_OK) return r;
+    // the partials of an earlier call are stale but harmless: every CTA rewrites its rows before they are merged
+    LinArgs a{};
+    a.W = W; a.N = V; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
+    a.epi = EPI_HEAD; a.scale = logit_scale; a.head_part = (float4*)scratch;
+    a.logits_dbg = logits; a.ld_dbg = V;
+    r = op_linear_common(dtype, a, (cudaStream_t)stream);
     if (r != KG_OK) return r;
     op_head_final_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(a.head_part, sm_count(), M, tok, p);
     CK(cudaGetLastError());
