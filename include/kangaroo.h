@@ -193,10 +193,10 @@ int kg_op_lm_head(int32_t dtype, const void* W_head_dev, int32_t V, int32_t K, c
  * a deployment convenience).  It is for callers that cannot obtain device memory at the time of the call -
  * code running while a memory pool is frozen or exhausted, inside a plugin whose host forbids cudaMalloc, or
  * in an error path that must still produce a token.  The per-CTA partial results that kg_op_lm_head keeps in
- * `scratch_dev` live here in a 64 KB array that is part of the library image, so every GPU that loads the
- * library holds those 64 KB until the process exits.
- * Limits: M <= KG_M_MAX rows and a device with at most 256 SMs (one partial per SM and row); anything larger
- * returns KG_E_LIMIT.  V and K are not limited: W, x and the outputs remain caller memory.
+ * `scratch_dev` (per-CTA partial results, and the repacked copy of the input rows) lives here in a 592 KB array
+ * that is part of the library image, so every GPU that loads the library holds those 592 KB until the process exits.
+ * Limits: M <= KG_M_MAX rows, K <= 8192 and a device with at most 256 SMs; anything larger returns KG_E_LIMIT.
+ * V is not limited: W, x and the outputs remain caller memory.
  * The first call on each device looks up the array's device address (no allocation); make that first call
  * outside any stream capture.  All calls share the one array: two calls whose kernels overlap on the GPU
  * (different streams, no ordering between them) race on it and give wrong results; calls ordered on one

@@ -65,6 +65,32 @@ __global__ void fill_tokens_kernel(int* out, uint64_t base, int count, int vocab
         out[i] = (int)(mix64(base + (uint64_t)i) % (uint64_t)vocab);
 }
 
+// fp32 rows -> packed rows (scaled by gain) + per-slice sums of squares, sliced over the columns exactly as the
+// CTAs of the decode kernel slice an operator's output (slice c = columns [K c / n, K (c+1) / n)).
+__global__ void pack_rows_kernel(const float* x, int ldx, int M, int K, const float* gain, unsigned char* xpk, int ldpk,
+                                 float* ssq, int nslices) {
+    __shared__ float sred[8];
+    const int cta = blockIdx.x;
+    const int k0 = (int)((unsigned)K * (unsigned)cta / (unsigned)nslices), k1 = (int)((unsigned)K * (unsigned)(cta + 1) / (unsigned)nslices);
+    for (int m = 0; m < M; ++m) {
+        float ss = 0.f;
+        for (int k = k0 + threadIdx.x; k < k1; k += blockDim.x) {
+            const float v = x[(size_t)m * ldx + k];
+            ss += v * v;
+            pk_store(xpk + (size_t)m * ldpk, k, gain ? v * gain[k] : v);
+        }
+        ss = warp_sum(ss);
+        if ((threadIdx.x & 31) == 0) sred[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        if (threadIdx.x == 0 && ssq) {
+            float t = 0.f;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sred[w];
+            ssq[(size_t)m * nslices + cta] = t;
+        }
+        __syncthreads();
+    }
+}
+
 enum { TID_EMBED = 1, TID_HEAD = 2, TID_PROMPT = 3, TID_HIDDEN = 4, TID_GFINAL = 6, TID_DRAFT = 7, TID_LAYER_BASE = 100 };
 enum { K_WQKV = 0, K_WO = 1, K_WGATE = 2, K_WUP = 3, K_WDOWN = 4, K_G1 = 5, K_G2 = 6, K_KCACHE = 8, K_VCACHE = 9 };
 inline uint64_t layer_tid(int layer, int k) { return (uint64_t)TID_LAYER_BASE + 16ull * (uint64_t)layer + (uint64_t)k; }
@@ -72,6 +98,7 @@ inline uint64_t layer_tid(int layer, int k) { return (uint64_t)TID_LAYER_BASE + 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
+    size_t off_hApk, off_hBpk, off_attnpk, off_actpk, off_featApk, off_featDpk, off_abufpk, off_ssqA, off_ssqB, off_ssqF, off_ssqAb;
     size_t off_layers, off_pt, off_kc, off_vc, off_h, off_feat, off_abuf, off_qkv, off_attn, off_act, off_po, off_ml,
         off_cnt, off_hp, off_dbgd, off_dbgv, off_out, off_S, off_rlog, off_prompt, off_st, off_bar;
     size_t off_embed, off_head, off_gfinal;
@@ -90,6 +117,7 @@ bool valid_config(const kg_config* c) {
     if (c->gamma_max < 1 || c->gamma_max > KG_GAMMA_MAX) return false;
     if (c->page_size < 1 || c->max_seq < 2) return false;
     if (c->n_heads > 256) return false;
+    if (c->vocab > (1 << 20) || c->d_ffn > (1 << 20)) return false;      // rows x CTAs must fit 32 bits
     // the plain path stages all rows of an operand in shared memory
     const int kmax = c->d_ffn > c->d_model ? c->d_ffn : c->d_model;
     const bool plain_somewhere = c->dtype == KG_F32 || (c->d_model % 16) || (c->d_ffn % 16);
@@ -118,6 +146,17 @@ Layout make_layout(const kg_config* c, int own_weights, int nctas) {
     L.off_qkv = take(4 * KG_M_MAX * 3 * d);
     L.off_attn = take(4 * KG_M_MAX * d);
     L.off_act = take(4 * KG_M_MAX * F);
+    L.off_hApk = take(4 * KG_M_MAX * d);
+    L.off_hBpk = take(4 * KG_M_MAX * d);
+    L.off_attnpk = take(4 * KG_M_MAX * d);
+    L.off_actpk = take(4 * KG_M_MAX * F);
+    L.off_featApk = take(4 * (KG_M_MAX + 1) * d);
+    L.off_featDpk = take(4 * (KG_M_MAX + 1) * d);
+    L.off_abufpk = take(4 * 2 * d);
+    L.off_ssqA = take(4 * (size_t)KG_M_MAX * nctas);
+    L.off_ssqB = take(4 * (size_t)KG_M_MAX * nctas);
+    L.off_ssqF = take(4 * (size_t)(KG_M_MAX + 1) * nctas);
+    L.off_ssqAb = take(4 * (size_t)2 * nctas);
     L.off_po = take(4 * (size_t)KG_M_MAX * H * S_CAP * hd);
     L.off_ml = take(4 * (size_t)KG_M_MAX * H * S_CAP * 2);
     L.off_cnt = take(4 * H);
@@ -202,7 +241,7 @@ extern "C" size_t kg_workspace_bytes(const kg_config* cfg, int own_weights) {
 
 template <typename WT>
 static int launch_program(kg_model* m, const Program& pg) {
-    CK(cudaMemsetAsync(m->dev.bar, 0, sizeof(unsigned), m->stream));
+    CK(cudaMemsetAsync(m->dev.bar, 0, BAR_BYTES, m->stream));
     Program p = pg;
     p.force_simple = m->force_simple;
     void* args[] = {(void*)&m->dev, (void*)&p};
@@ -299,6 +338,13 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     D.qkv = (float*)P(lay.off_qkv); D.attn = (float*)P(lay.off_attn); D.act = (float*)P(lay.off_act);
     D.att_po = (float*)P(lay.off_po); D.att_ml = (float*)P(lay.off_ml); D.att_cnt = (unsigned*)P(lay.off_cnt);
     D.head_part = (float4*)P(lay.off_hp);
+    D.hA_pk = (unsigned char*)P(lay.off_hApk); D.hB_pk = (unsigned char*)P(lay.off_hBpk);
+    D.attn_pk = (unsigned char*)P(lay.off_attnpk); D.act_pk = (unsigned char*)P(lay.off_actpk);
+    D.featA_pk = (unsigned char*)P(lay.off_featApk); D.featD_pk = (unsigned char*)P(lay.off_featDpk);
+    D.abuf_pk = (unsigned char*)P(lay.off_abufpk);
+    D.ssq_hA = (float*)P(lay.off_ssqA); D.ssq_hB = (float*)P(lay.off_ssqB);
+    D.ssq_feat = (float*)P(lay.off_ssqF); D.ssq_abuf = (float*)P(lay.off_ssqAb);
+    D.dm.stream = (cfg->dtype == KG_BF16 && cfg->d_model % 16 == 0 && cfg->d_ffn % 16 == 0) ? 1 : 0;
     D.dbg_draft = cfg->debug_logits ? (float*)P(lay.off_dbgd) : nullptr;
     D.dbg_verify = cfg->debug_logits ? (float*)P(lay.off_dbgv) : nullptr;
     D.out_tokens = (int*)P(lay.off_out); D.S = (int*)P(lay.off_S); D.round_log = (int*)P(lay.off_rlog);
@@ -662,6 +708,11 @@ extern "C" int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t
         }
     }
     fill_f32_kernel<<<64, 256, 0, s>>>(m->dev.feat, stream_base(seed, TID_HIDDEN), (uint64_t)(KG_M_MAX + 1) * c.d_model, one);
+    if (m->dev.dm.stream) {
+        const int d = c.d_model;
+        pack_rows_kernel<<<m->nctas, 256, 0, s>>>(m->dev.feat, d, KG_M_MAX + 1, d, m->layers_host[c.n_layers].g1, m->dev.featA_pk, d * 4, m->dev.ssq_feat, m->nctas);
+        pack_rows_kernel<<<m->nctas, 256, 0, s>>>(m->dev.feat, d, KG_M_MAX + 1, d, m->layers_host[c.exit_layer].g1, m->dev.featD_pk, d * 4, m->dev.ssq_feat, m->nctas);
+    }
     CK(cudaGetLastError());
     // tokens: x_0 and the drafts
     const uint64_t tb = stream_base(seed, TID_DRAFT);
@@ -689,7 +740,8 @@ extern "C" int kg_debug_force_simple(kg_model* m, int on) {
 // ------------------------------------------------------------------------------------ single operators
 namespace {
 
-struct OpScratch { size_t off_hp, off_po, off_ml, off_cnt, off_pt, total; };
+constexpr int OP_K_MAX = 32768;               // longest input row the single-operator entry points pack into scratch
+struct OpScratch { size_t off_hp, off_po, off_ml, off_cnt, off_pt, off_xpk, off_ssq, total; };
 OpScratch op_layout() {
     OpScratch s; size_t o = 0;
     auto take = [&](size_t b) { size_t r = o; o = align_up(o + b, 256); return r; };
@@ -697,16 +749,18 @@ OpScratch op_layout() {
     s.off_po = take(4 * (size_t)KG_M_MAX * S_CAP * 8192);
     s.off_ml = take(4 * (size_t)KG_M_MAX * 256 * S_CAP * 2);
     s.off_cnt = take(4 * 256);
+    s.off_xpk = take(4 * (size_t)KG_M_MAX * OP_K_MAX);
+    s.off_ssq = take(4 * (size_t)KG_M_MAX * 1024);
     s.total = o;
     return s;
 }
 
 template <typename WT>
-__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int force_simple) {
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int stream) {
     extern __shared__ __align__(128) char smem[];
     Ctx c;
     ctx_init(c, smem, nullptr, nullptr, false);
-    const bool ok = linear_op<WT>(a, c, force_simple != 0);
+    const bool ok = linear_op<WT>(a, c, stream != 0);
     if (!ok && c.producer) ring_drain(c);
 }
 __global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* tok, float* p) {
@@ -733,18 +787,24 @@ extern "C" size_t kg_op_scratch_bytes(void) { return op_layout().total; }
 
 extern "C" int kg_debug_force_simple_ops(int on) { g_force_simple_ops = on ? 1 : 0; return KG_OK; }
 
-static int op_linear_common(int32_t dtype, LinArgs& a, cudaStream_t s) {
+// xpk / ssq: scratch for the packed copy of the input rows (xpk_k_max = longest row it holds) and their sums of squares
+static int op_linear_common(int32_t dtype, LinArgs& a, unsigned char* xpk, int xpk_k_max, float* ssq, cudaStream_t s) {
     if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
-    if (a.M < 1 || a.M > KG_M_MAX || a.N < 1 || a.K < 8 || (a.K % 8)) return KG_E_ARG;
+    if (a.M < 1 || a.M > KG_M_MAX || a.N < 1 || a.N > (1 << 20) || a.K < 8 || (a.K % 8)) return KG_E_ARG;
     const bool plain = dtype == KG_F32 || g_force_simple_ops || (a.K % 16);
     if (plain && (size_t)a.K * a.M * 4 > (size_t)SIMPLE_XS_BYTES) return KG_E_ARG;
     const int nctas = sm_count();
+    if (!plain) {
+        if (a.K > xpk_k_max || nctas > 1024) return KG_E_LIMIT;
+        pack_rows_kernel<<<nctas, 256, 0, s>>>(a.x, a.ldx, a.M, a.K, a.gain, xpk, a.K * 4, a.gain ? ssq : nullptr, nctas);
+        a.xpk = xpk; a.ldpk = a.K * 4; a.ssq_in = a.gain ? ssq : nullptr;
+    }
     if (dtype == KG_BF16) {
         if (set_smem(op_linear_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, g_force_simple_ops);
+        op_linear_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, plain ? 0 : 1);
     } else {
         if (set_smem(op_linear_kernel<float>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, g_force_simple_ops);
+        op_linear_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, 0);
     }
     CK(cudaGetLastError());
     return KG_OK;
@@ -759,7 +819,8 @@ extern "C" int kg_op_linear(int32_t dtype, const void* W, const void* W2, int32_
     a.W = W; a.W2 = swiglu ? W2 : nullptr; a.N = N; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
     a.resid = resid; a.ldr = N; a.out = out; a.ldo = N;
     a.epi = swiglu ? EPI_SWIGLU : (resid ? EPI_RESID : EPI_STORE);
-    return op_linear_common(dtype, a, (cudaStream_t)stream);
+    OpScratch sc = op_layout();
+    return op_linear_common(dtype, a, (unsigned char*)scratch + sc.off_xpk, OP_K_MAX, (float*)((char*)scratch + sc.off_ssq), (cudaStream_t)stream);
 }
 
 extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K, const float* x, int32_t M,
@@ -772,7 +833,7 @@ extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K,
     a.W = W; a.N = V; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
     a.epi = EPI_HEAD; a.scale = logit_scale; a.head_part = (float4*)((char*)scratch + sc.off_hp);
     a.logits_dbg = logits; a.ld_dbg = V;
-    int r = op_linear_common(dtype, a, (cudaStream_t)stream);
+    int r = op_linear_common(dtype, a, (unsigned char*)scratch + sc.off_xpk, OP_K_MAX, (float*)((char*)scratch + sc.off_ssq), (cudaStream_t)stream);
     if (r != KG_OK) return r;
     op_head_final_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(a.head_part, sm_count(), M, tok, p);
     CK(cudaGetLastError());
@@ -784,8 +845,12 @@ extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K,
 // scratch is a fixed array inside the library image instead of caller memory.
 namespace {
 constexpr int NOALLOC_MAX_CTAS = 256;                        // CTAs (one per SM) the static scratch has room for
+constexpr int NOALLOC_MAX_K = 8192;                          // longest input row it can pack
 constexpr int NOALLOC_MAX_DEVICES = 64;
-static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(float4) * NOALLOC_MAX_CTAS * KG_M_MAX];   // 64 KB
+constexpr size_t NOALLOC_OFF_XPK = sizeof(float4) * NOALLOC_MAX_CTAS * KG_M_MAX;                 // head partials first: 64 KB
+constexpr size_t NOALLOC_OFF_SSQ = NOALLOC_OFF_XPK + 4 * (size_t)KG_M_MAX * NOALLOC_MAX_K;        // packed input rows: 512 KB
+constexpr size_t NOALLOC_BYTES = NOALLOC_OFF_SSQ + 4 * (size_t)KG_M_MAX * NOALLOC_MAX_CTAS;       // sums of squares: 16 KB
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
 void* g_noalloc_addr[NOALLOC_MAX_DEVICES] = {nullptr};
 
 // Device address of the static scratch on the current device.  In host code the array's name is only a
@@ -808,7 +873,7 @@ extern "C" int kg_op_lm_head_noalloc(int32_t dtype, const void* W, int32_t V, in
                                      const float* gain, float eps, float logit_scale,
                                      int32_t* tok, float* p, float* logits, void* stream) {
     if (!W || !x || !tok || !p) return KG_E_ARG;
-    if (M > KG_M_MAX || sm_count() > NOALLOC_MAX_CTAS) return KG_E_LIMIT;
+    if (M > KG_M_MAX || K > NOALLOC_MAX_K || sm_count() > NOALLOC_MAX_CTAS) return KG_E_LIMIT;
     void* scratch = nullptr;
     int r = noalloc_scratch(&scratch);
     if (r != KG_OK) return r;
@@ -817,7 +882,8 @@ extern "C" int kg_op_lm_head_noalloc(int32_t dtype, const void* W, int32_t V, in
     a.W = W; a.N = V; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
     a.epi = EPI_HEAD; a.scale = logit_scale; a.head_part = (float4*)scratch;
     a.logits_dbg = logits; a.ld_dbg = V;
-    r = op_linear_common(dtype, a, (cudaStream_t)stream);
+    r = op_linear_common(dtype, a, (unsigned char*)scratch + NOALLOC_OFF_XPK, NOALLOC_MAX_K, (float*)((char*)scratch + NOALLOC_OFF_SSQ),
+                         (cudaStream_t)stream);
     if (r != KG_OK) return r;
     op_head_final_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(a.head_part, sm_count(), M, tok, p);
     CK(cudaGetLastError());

@@ -5,7 +5,7 @@
 // (cta, nctas) and a grid-wide barrier separates dependent operators.  The same operators are
 // also wrapped one-by-one in small kernels for unit tests.
 //
-// A CTA has 16 consumer warps and one producer warp.  The decode step is bound by HBM bandwidth:
+// A CTA has 8 consumer warps and one producer warp.  The decode step is bound by HBM bandwidth:
 // every weight byte is read exactly once per pass.  The producer warp streams this CTA's share of
 // every weight matrix of a pass through a ring of shared-memory slots with bulk asynchronous
 // copies (cp.async.bulk + mbarrier transaction counts); because weights do not depend on
@@ -21,7 +21,10 @@
 
 // Timeline hook for profiling builds (a translation unit may define it before including this file).
 #ifndef KG_PROBE
-#define KG_PROBE(slot) do { } while (0)
+#define KG_PROBE(tag) do { } while (0)
+#endif
+#ifndef KG_PROBE_INIT
+#define KG_PROBE_INIT() do { } while (0)
 #endif
 
 namespace kg {
@@ -49,6 +52,8 @@ constexpr int WORK_BYTES = SMEM_TOTAL - WORK_OFF;       // activations, reductio
 constexpr int SC_ROWS = 256;                            // rows whose accumulators live in shared memory at once
 constexpr int SIMPLE_XS_BYTES = WORK_BYTES - 4096;      // activation staging of the plain path
 
+constexpr int BAR_RELEASE = 32;                          // word index of the grid barrier's release word (its own 128-byte line)
+constexpr int BAR_BYTES = 256;
 constexpr unsigned long long WAIT_TIMEOUT_CLK = 6000000000ull;   // ~3 s at 1.9 GHz
 
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_HEAD = 3 };
@@ -63,6 +68,7 @@ struct Dims {
     int L, d, H, hd, F, V, l;
     float eps, theta, logit_scale;
     int max_seq, page_size, n_pages, gamma_max, debug;
+    int stream;         // 1: linear operators take the streamed tensor-core path (bf16, d and F multiples of 16)
 };
 
 // Device-resident sequence / round state (one int-sized field per line of the method's notation).
@@ -97,6 +103,17 @@ struct Dev {
     float* qkv;                    // [M_MAX][3d]
     float* attn;                   // [M_MAX][d]
     float* act;                    // [M_MAX][F]
+    // packed copies (streamed path; row = 4 bytes per element) and per-CTA sums of squares [row][nctas]
+    unsigned char* hA_pk;          // [M_MAX][d]   residual stream scaled for the next QKV / the LM head
+    unsigned char* hB_pk;          // [M_MAX][d]   residual stream after attention scaled for the SwiGLU pair
+    unsigned char* attn_pk;        // [M_MAX][d]
+    unsigned char* act_pk;         // [M_MAX][F]
+    unsigned char* featA_pk;       // [M_MAX+1][d] early features scaled by the adapter's input gain
+    unsigned char* featD_pk;       // [M_MAX+1][d] early features scaled by the first deep layer's gain
+    unsigned char* abuf_pk;        // [2][d]       adapter output scaled by its last gain
+    float* ssq_hA; float* ssq_hB;  // [M_MAX][nctas]
+    float* ssq_feat;               // [M_MAX+1][nctas]
+    float* ssq_abuf;               // [2][nctas]
     float* att_po;                 // [M_MAX][H][S_CAP][hd] split partial outputs
     float* att_ml;                 // [M_MAX][H][S_CAP][2]  split partial (max, sum)
     unsigned* att_cnt;             // [H] arrival counters
@@ -114,7 +131,6 @@ struct Ctrl {
     unsigned long long full[RING];     // producer -> consumers: slot filled (transaction count)
     unsigned long long empty[RING];    // consumers -> producer: slot drained (one arrival per consumer warp)
     unsigned long long mail;           // consumers -> producer: head_tok / head_p hold a new result
-    unsigned long long xfull;          // activation rows of a k phase have landed in shared memory
     int abort;                         // a bounded wait of this CTA gave up
     int sync_ok;
     int att_last;
@@ -134,7 +150,6 @@ struct Ctx {
     int slot; unsigned phase;      // ring cursor of this thread's role
     unsigned issued;               // producer: stages issued so far
     unsigned mail_phase;           // producer: parity of the next result it waits for
-    unsigned x_phase;              // consumers: parity of the next activation stage
 };
 
 // ------------------------------------------------------------------------------------ helpers
@@ -243,11 +258,11 @@ __device__ __forceinline__ void ctx_init(Ctx& c, char* smem, State* st, unsigned
     c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
     c.ctl = reinterpret_cast<Ctrl*>(smem); c.grid = grid;
     c.producer = threadIdx.x >= NTHREADS;
-    c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0; c.x_phase = 0;
+    c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0;
+    KG_PROBE_INIT();
     if (threadIdx.x == 0) {
         for (int i = 0; i < RING; ++i) { mbar_init(&c.ctl->full[i], 1); mbar_init(&c.ctl->empty[i], NWARPS); }
         mbar_init(&c.ctl->mail, 1);
-        mbar_init(&c.ctl->xfull, 1);
         c.ctl->abort = 0; c.ctl->sync_ok = 1; c.ctl->att_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -263,16 +278,23 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
     cta_sync();
     KG_PROBE(1);
     if (threadIdx.x == 0) {
+        // bar[0] counts arrivals (monotonic over the launch); bar[BAR_RELEASE] is written once per barrier
+        // by the last CTA to arrive, so the waiting CTAs poll a word nobody else is updating
         c.bar_target += (unsigned)c.nctas;
+        const unsigned gen = c.bar_target;
         __threadfence();
-        atomicAdd(c.bar, 1u);
+        const unsigned prev = atomicAdd(c.bar, 1u);
         int ok = 1;
-        long long t0 = clock64();
-        unsigned spins = 0;
-        while ((int)(ld_acquire_u32(c.bar) - c.bar_target) < 0) {
-            if (((++spins) & 63u) == 0u) {
-                if (*(volatile int*)&c.st->status != 0) { ok = 0; break; }
-                if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
+        if (prev + 1u == gen) {
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(c.bar + BAR_RELEASE), "r"(gen) : "memory");
+        } else {
+            const long long t0 = clock64();
+            unsigned spins = 0;
+            while ((int)(ld_acquire_u32(c.bar + BAR_RELEASE) - gen) < 0) {
+                if (((++spins) & 63u) == 0u) {
+                    if (*(volatile int*)&c.st->status != 0) { ok = 0; break; }
+                    if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
+                }
             }
         }
         if (*(volatile int*)&c.st->status != 0) ok = 0;
@@ -296,17 +318,41 @@ __device__ __forceinline__ void rope_cs(const Dev& D, int pos, int i, float& cs,
 }
 
 // ------------------------------------------------------------------------------------ linear operator
+// A packed copy of activation rows: the row is cut into k16 blocks of 64 bytes; the 16 bytes at
+// blk*64 + tt*16 hold {hi(k), hi(k+8), lo(k), lo(k+8)} for k = 16 blk + 2 tt, each a pair of bf16
+// (elements k, k+1) with x * gain = hi + lo.  This is the B operand fragment order of the MMA, so a
+// consumer lane fetches its fragments with plain 8- or 16-byte loads.  The operator that produces a
+// row writes it once, in this form, for the operator that reads it.
+struct PkOut { const float* gain; unsigned char* ptr; };   // gain == null: unscaled
+
+// byte offset of the hi half of element k inside a packed row; the lo half sits 8 bytes further
+__device__ __forceinline__ size_t pk_off(int k) {
+    return (size_t)(k >> 4) * 64 + (size_t)(((k & 7) >> 1) * 16 + ((k >> 3) & 1) * 4 + (k & 1) * 2);
+}
+__device__ __forceinline__ void pk_store(unsigned char* row, int k, float v) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
+    unsigned char* p = row + pk_off(k);
+    *reinterpret_cast<__nv_bfloat16*>(p) = h;
+    *reinterpret_cast<__nv_bfloat16*>(p + 8) = l;
+}
+
 struct LinArgs {
     const void* W; const void* W2;   // [N, K]; W2 != null: SwiGLU pair (gate, up)
     int N, K;
-    const float* x; int ldx; int M;  // activation rows (fp32, written earlier in this kernel)
-    const float* gain; float eps;    // RMSNorm gain (null: no norm)
+    int M;                           // activation rows
+    const float* x; int ldx;         // plain path: fp32 rows (written earlier in this kernel)
+    const float* gain; float eps;    // RMSNorm gain of the input (null: no norm)
+    const unsigned char* xpk; int ldpk;   // streamed path: packed rows, already multiplied by the gain; bytes per row
+    const float* ssq_in;             // streamed path with norm: [M][nctas] partial sums of squares of the input rows
     const float* resid; int ldr;     // EPI_RESID
-    float* out; int ldo;
+    float* out; int ldo;             // fp32 output rows (streamed path: nullable)
     int epi;
     float scale;                     // EPI_HEAD: logit scale
     float4* head_part;               // EPI_HEAD: [nctas][M_MAX]
     float* logits_dbg; int ld_dbg;   // EPI_HEAD, optional
+    PkOut pk[2]; int ldpk_out;       // streamed path: packed copies of the output rows for the operators that read them
+    float* ssq_out;                  // streamed path: [M][nctas] partial sums of squares of the output rows (nullable)
 };
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
@@ -341,10 +387,9 @@ __device__ __forceinline__ void head_merge(HeadStat& a, float zmax, float sum, i
 //   V = 4  (M <= 4):  columns 0-3 carry hi, columns 4-7 lo of rows 0-3: one MMA per k16-step;
 //   V = 8  (M <= 8):  hi and lo are two MMAs;
 //   V = 16 (M <= 16): two column tiles, hi and lo: four MMAs.
-// Each of the 8 warps owns a fixed slice of the phase's k range; its B fragments are built once
-// per phase (from an fp32 copy of the activation rows that a bulk copy placed in shared memory one
-// phase ahead) and stay in registers for every row group, so the steady state touches shared
-// memory only for the weights.  After a stage pair the 8 partial sums of each (weight row,
+// Each of the 8 warps owns a fixed slice of the phase's k range; its B fragments are loaded once
+// per phase from the packed activation rows in global memory (L2) and stay in registers for every
+// row group, so the steady state touches shared memory only for the weights.  After a stage pair the 8 partial sums of each (weight row,
 // activation row) are added in warp order into the per-row accumulators in shared memory.
 template <int V> struct LinGeom {
     static constexpr int NS = V == 16 ? 8 : 16;           // k16-steps per warp and stage
@@ -362,8 +407,8 @@ struct LinPlan {
 
 __device__ __forceinline__ LinPlan make_plan(const LinArgs& a, int cta, int nctas) {
     LinPlan p;
-    p.u0 = (int)((long long)a.N * cta / nctas);
-    p.u1 = (int)((long long)a.N * (cta + 1) / nctas);
+    p.u0 = (int)((unsigned)a.N * (unsigned)cta / (unsigned)nctas);          // N * nctas < 2^32 (checked on the host)
+    p.u1 = (int)((unsigned)a.N * (unsigned)(cta + 1) / (unsigned)nctas);
     p.sc_units = a.W2 ? SC_ROWS / 2 : SC_ROWS;
     p.plen = a.M <= 8 ? LinGeom<8>::PLEN : LinGeom<16>::PLEN;
     p.nph = (a.K + p.plen - 1) / p.plen;
@@ -426,90 +471,149 @@ __device__ __forceinline__ void split_hi_lo(float2 v, unsigned& hi, unsigned& lo
     lo = *reinterpret_cast<const unsigned*>(&l);
 }
 
-// Consumer warp 0: start the bulk copies of the activation rows (and the gain) of one k phase.
-__device__ __forceinline__ void issue_x_phase(const LinArgs& a, Ctx& c, char* xs, int p0, int len, int xrow_bytes, int gain_row) {
-    const int lane = threadIdx.x & 31;
-    const int nrows = a.M + (a.gain ? 1 : 0);
-    if (lane == 0) mbar_arrive_expect_tx(&c.ctl->xfull, (unsigned)(nrows * len * 4));
-    asm volatile("fence.proxy.async;" ::: "memory");     // the rows were written with ordinary stores
-    __syncwarp();
-    if (lane < a.M) bulk_g2s(xs + (size_t)lane * xrow_bytes, a.x + (size_t)lane * a.ldx + p0, (unsigned)(len * 4), &c.ctl->xfull);
-    if (lane == M_MAX && a.gain) bulk_g2s(xs + (size_t)gain_row * xrow_bytes, a.gain + p0, (unsigned)(len * 4), &c.ctl->xfull);
+// Shared-memory work area of the streamed path (floats, from WORK_OFF).
+constexpr int LW_RED = 0;                                 // [2][NWARPS][16][8] partial sums of a stage pair
+constexpr int LW_ACC = LW_RED + 2 * NWARPS * 128;         // [SC_ROWS][MP] row accumulators
+constexpr int LW_RS = LW_ACC + SC_ROWS * MP;              // [M_MAX] 1/rms of the input rows
+constexpr int LW_RSP = LW_RS + M_MAX;                     // [M_MAX][16] partial sums of squares of the input rows
+constexpr int LW_SSW = LW_RSP + M_MAX * 16;               // [NWARPS][M_MAX] sums of squares of the output rows
+constexpr int PRE_NU = 64;                                // residual / gain values are prefetched for up to this many units
+constexpr int LW_PRES = LW_SSW + NWARPS * M_MAX;          // [M_MAX][PRE_NU] residual values
+constexpr int LW_PREG = LW_PRES + M_MAX * PRE_NU;         // [2][PRE_NU] gains of the packed outputs
+constexpr int LW_END = LW_PREG + 2 * PRE_NU;
+static_assert(LW_END * 4 <= WORK_BYTES, "linear work area too large");
+
+__device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+
+// Epilogue of the streamed path for everything but the LM head: turns the accumulators of nu output
+// units x M rows (acc_s, 1/rms in rs) into fp32 rows, packed copies and per-CTA sums of squares.
+// Thread (r, m): m = tid mod 2^ceil(log2 M), so that the lanes of a warp that share m can add their
+// squares by shuffles in a fixed order.  Every consumer thread calls it; ssq_acc (threads < M)
+// accumulates over superchunks.
+__device__ __forceinline__ void emit_rows(const LinArgs& a, float* wk, int sc0, int nu, bool prefetched, float& ssq_acc) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int M = a.M;
+    const float* acc_s = wk + LW_ACC;
+    const float* rs = wk + LW_RS;
+    float* ssw = wk + LW_SSW;
+    const int sh = M <= 1 ? 0 : (M <= 2 ? 1 : (M <= 4 ? 2 : (M <= 8 ? 3 : 4)));
+    const int mp = 1 << sh;
+    const int m = tid & (mp - 1);
+    float ssl = 0.f;
+    if (m < M) {
+        for (int r = tid >> sh; r < nu; r += NTHREADS >> sh) {
+            float v;
+            if (a.epi == EPI_SWIGLU) {
+                const int srow = (r >> 3) * 16 + (r & 7);
+                v = silu_f(acc_s[(size_t)srow * MP + m] * rs[m]) * (acc_s[(size_t)(srow + 8) * MP + m] * rs[m]);
+            } else {
+                v = acc_s[(size_t)r * MP + m] * rs[m];
+                if (a.epi == EPI_RESID)
+                    v += prefetched ? wk[LW_PRES + m * PRE_NU + r] : ldcg_f(a.resid + (size_t)m * a.ldr + sc0 + r);
+            }
+            const int row = sc0 + r;
+            if (a.out) a.out[(size_t)m * a.ldo + row] = v;
+            ssl += v * v;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                if (a.pk[q].ptr) {
+                    float pv = v;
+                    if (a.pk[q].gain) pv *= prefetched ? wk[LW_PREG + q * PRE_NU + r] : __ldg(a.pk[q].gain + row);
+                    pk_store(a.pk[q].ptr + (size_t)m * a.ldpk_out, row, pv);
+                }
+            }
+        }
+    }
+    if (a.ssq_out) {
+        for (int o = 16; o >= mp; o >>= 1) ssl += __shfl_xor_sync(0xffffffffu, ssl, o);
+        if (lane < mp) ssw[warp * M_MAX + lane] = ssl;
+        cta_sync();
+        if (tid < M) {
+            float sres = 0.f;
+            for (int w = 0; w < NWARPS; ++w) sres += ssw[w * M_MAX + tid];
+            ssq_acc += sres;
+        }
+    }
 }
 
 template <int V>
 __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
     using G = LinGeom<V>;
     constexpr int NS = G::NS, FR = G::FR, NACC = G::NACC;
-    constexpr int XRB = G::PLEN * 4 + 32;                                  // byte stride of a staged activation row
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int M = a.M, K = a.K;
     const bool dual = a.W2 != nullptr;
     const LinPlan pl = make_plan(a, c.cta, c.nctas);
 
-    char* xs = c.smem + WORK_OFF;                                          // [V + 1][XRB] fp32 activation rows of a phase, then the gain
-    float* red = reinterpret_cast<float*>(xs + (V + 1) * XRB);             // [2 | 1][NWARPS][NACC][16][8] partial sums
-    float* acc_s = red + 2 * NWARPS * 128;                                 // [SC_ROWS][MP]
-    float* ssw = acc_s + SC_ROWS * MP;                                     // [NWARPS][M_MAX] sums of squares
-    float* rs = ssw + NWARPS * M_MAX;                                      // [M_MAX] 1/rms
+    float* wk = reinterpret_cast<float*>(c.smem + WORK_OFF);
+    float* red = wk + LW_RED;
+    float* acc_s = wk + LW_ACC;
+    float* rs = wk + LW_RS;
     const char* ring = c.smem + RING_OFF;
 
     HeadStat hs[2];                                                        // EPI_HEAD: this warp tracks rows warp, warp + 8
     hs[0].zmax = hs[1].zmax = 0.f; hs[0].sum = hs[1].sum = 0.f; hs[0].arg = hs[1].arg = 0;
     bool ok = true;
     int buf = 0;
+    float ssq_acc = 0.f;
     KG_PROBE(10);
-    // activation row(s) this lane converts: V = 4: row g & 3 (hi for g < 4, lo otherwise); else rows g (and g + 8)
-    const int xrow = V == 4 ? (g & 3) : g;
-    float ssq[NACC];
+
+    // ---- fetched now, used in the epilogue: the input rows' sums of squares, residual values, output gains
+    const int nu0 = min(pl.u1 - pl.u0, pl.sc_units);
+    const bool prefetched = nu0 <= PRE_NU;
+    if (a.ssq_in) {
+        // thread (m, j) adds the partial sums of CTAs j, j + 16, ... of row m
+        const int m = tid >> 4, j = tid & 15;
+        float part = 0.f;
+        if (m < M) for (int q = j; q < c.nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * c.nctas + q);
+        wk[LW_RSP + tid] = part;
+    }
+    if (prefetched && a.epi != EPI_HEAD) {
+        if (a.epi == EPI_RESID)
+            for (int i = tid; i < M * nu0; i += NTHREADS) cp_async4(wk + LW_PRES + (i / nu0) * PRE_NU + i % nu0, a.resid + (size_t)(i / nu0) * a.ldr + pl.u0 + i % nu0);
 #pragma unroll
-    for (int n = 0; n < NACC; ++n) ssq[n] = 0.f;
+        for (int q = 0; q < 2; ++q)
+            if (a.pk[q].ptr && a.pk[q].gain)
+                for (int i = tid; i < nu0; i += NTHREADS) cp_async4(wk + LW_PREG + q * PRE_NU + i, a.pk[q].gain + pl.u0 + i);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+
+    // this lane's rows of the packed input: V = 4: row g & 3 (hi for g < 4, lo for g >= 4); else rows g (and g + 8)
+    const int xrow = V == 4 ? (g & 3) : g;
+    const unsigned char* xlane = a.xpk + (size_t)xrow * a.ldpk + (size_t)warp * NS * 64 + t * 16 + (V == 4 ? (g >> 2) * 8 : 0);
 
     for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
         const int sc1 = min(pl.u1, sc0 + pl.sc_units);
         const int nu = sc1 - sc0;
         const int ngrp = (nu + ST_ROWS - 1) / ST_ROWS;
         const int nst = dual ? 2 * ngrp : ngrp;
-        if (warp == 0) issue_x_phase(a, c, xs, 0, min(pl.plen, K), XRB, V);
         for (int ph = 0; ph < pl.nph; ++ph) {
             const int p0 = ph * pl.plen, len = min(pl.plen, K - p0);
             const int nsteps = len / 16;
-            // ---- B fragments of this warp's k slice: x * gain split into bf16 hi / lo
+            // ---- B fragments of this warp's k slice, kept in registers for every row group of the phase
             unsigned fr[NS][FR];
-            if (ok) ok = mbar_wait(c, &c.ctl->xfull, c.x_phase, 43);
-            c.x_phase ^= 1u;
 #pragma unroll
             for (int s = 0; s < NS; ++s) {
 #pragma unroll
                 for (int q = 0; q < FR; ++q) fr[s][q] = 0u;
-                const int st = warp * NS + s;
-                if (ok && st < nsteps) {
-                    const int kk = st * 16 + 2 * t;
-                    float2 g0 = make_float2(1.f, 1.f), g1 = g0;
-                    if (a.gain) {
-                        const float* gr = reinterpret_cast<const float*>(xs + (size_t)V * XRB) + kk;
-                        g0 = *reinterpret_cast<const float2*>(gr); g1 = *reinterpret_cast<const float2*>(gr + 8);
-                    }
+                if (warp * NS + s < nsteps) {
+                    const unsigned char* px = xlane + (size_t)(p0 / 16 + s) * 64;
+                    if (V == 4) {
+                        if (xrow < M) { const uint2 v = __ldcg(reinterpret_cast<const uint2*>(px)); fr[s][0] = v.x; fr[s][1] = v.y; }
+                    } else {
 #pragma unroll
-                    for (int n = 0; n < NACC; ++n) {
-                        const int m = xrow + 8 * n;
-                        if (m < M) {
-                            const float* xr = reinterpret_cast<const float*>(xs + (size_t)m * XRB) + kk;
-                            float2 u = *reinterpret_cast<const float2*>(xr), w = *reinterpret_cast<const float2*>(xr + 8);
-                            if (sc0 == pl.u0 && (V != 4 || g < 4)) ssq[n] += u.x * u.x + u.y * u.y + w.x * w.x + w.y * w.y;
-                            u.x *= g0.x; u.y *= g0.y; w.x *= g1.x; w.y *= g1.y;
-                            unsigned h0, l0, h8, l8;
-                            split_hi_lo(u, h0, l0);
-                            split_hi_lo(w, h8, l8);
-                            if (V == 4) { fr[s][0] = g < 4 ? h0 : l0; fr[s][1] = g < 4 ? h8 : l8; }
-                            else { fr[s][4 * n + 0] = h0; fr[s][4 * n + 1] = h8; fr[s][4 * n + 2] = l0; fr[s][4 * n + 3] = l8; }
+                        for (int n = 0; n < NACC; ++n) {
+                            if (xrow + 8 * n < M) {
+                                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(px + (size_t)(8 * n) * a.ldpk));
+                                fr[s][4 * n + 0] = v.x; fr[s][4 * n + 1] = v.y; fr[s][4 * n + 2] = v.z; fr[s][4 * n + 3] = v.w;
+                            }
                         }
                     }
                 }
             }
-            cta_sync();                                      // every warp has read the staged rows
-            if (warp == 0 && ph + 1 < pl.nph) issue_x_phase(a, c, xs, p0 + pl.plen, min(pl.plen, K - p0 - pl.plen), XRB, V);
             KG_PROBE(11);
             // ---- the row groups of this phase, two stages (16 weight rows) at a time
             const uint32_t a_lane = (uint32_t)((lane & 7) * ST_ROW_BYTES + (warp * NS * 16 + (lane >> 4) * 8) * 2);
@@ -587,37 +691,20 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
         }
         // ---- epilogue of this superchunk
         if (sc0 == pl.u0) {
-            // 1/rms per activation row: the four lanes sharing g hold the partial sums of row xrow (+ 8)
-#pragma unroll
-            for (int n = 0; n < NACC; ++n) {
-                float s = ssq[n];
-                s += __shfl_xor_sync(0xffffffffu, s, 1);
-                s += __shfl_xor_sync(0xffffffffu, s, 2);
-                if (t == 0 && (V != 4 || g < 4)) ssw[warp * M_MAX + xrow + 8 * n] = s;
-            }
-        }
-        cta_sync();
-        if (sc0 == pl.u0) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            cta_sync();
             if (tid < M_MAX) {
                 float r = 1.0f;
-                if (a.gain && tid < M) {
+                if (a.ssq_in && tid < M) {
                     float ss = 0.f;
-                    for (int w = 0; w < NWARPS; ++w) ss += ssw[w * M_MAX + tid];
+                    for (int j = 0; j < 16; ++j) ss += wk[LW_RSP + tid * 16 + j];
                     r = rsqrtf(ss / (float)K + a.eps);
                 }
                 rs[tid] = r;
             }
-            cta_sync();
         }
-        if (a.epi == EPI_SWIGLU) {
-            for (int idx = tid; idx < nu * M; idx += NTHREADS) {
-                const int fl_ = idx % nu, m = idx / nu;
-                const int srow = (fl_ >> 3) * 16 + (fl_ & 7);
-                const float vg = acc_s[(size_t)srow * MP + m] * rs[m];
-                const float vu = acc_s[(size_t)(srow + 8) * MP + m] * rs[m];
-                a.out[(size_t)m * a.ldo + sc0 + fl_] = silu_f(vg) * vu;
-            }
-        } else if (a.epi == EPI_HEAD) {
+        cta_sync();
+        if (a.epi == EPI_HEAD) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int m = warp + q * NWARPS;
@@ -642,15 +729,9 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                 }
             }
         } else {
-            for (int idx = tid; idx < nu * M; idx += NTHREADS) {
-                const int r = idx % nu, m = idx / nu;
-                float v = acc_s[(size_t)r * MP + m] * rs[m];
-                const size_t row = (size_t)(sc0 + r);
-                if (a.epi == EPI_RESID) v += ldcg_f(a.resid + (size_t)m * a.ldr + row);
-                a.out[(size_t)m * a.ldo + row] = v;
-            }
+            emit_rows(a, wk, sc0, nu, prefetched && sc0 == pl.u0, ssq_acc);
         }
-        cta_sync();                                  // acc_s and the staged rows are rewritten by the next superchunk / operator
+        cta_sync();                                  // acc_s is rewritten by the next superchunk / operator
         KG_PROBE(15);
     }
     if (a.epi == EPI_HEAD && lane == 0) {
@@ -660,6 +741,32 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
             if (m < M) a.head_part[(size_t)c.cta * M_MAX + m] = make_float4(hs[q].zmax, hs[q].sum, __int_as_float(hs[q].arg), 0.f);
         }
     }
+    if (a.epi != EPI_HEAD && a.ssq_out && tid < M) a.ssq_out[(size_t)tid * c.nctas + c.cta] = ssq_acc;
+}
+
+// Rows that do not come out of a linear operator (token embeddings): every CTA takes its slice of
+// the d columns, places the values where the epilogue expects accumulators and emits them like
+// an operator output (fp32 rows, packed copies, sums of squares).  value(m, e) is given by the caller.
+template <typename F>
+__device__ __forceinline__ void emit_plain_rows(LinArgs& a, Ctx& c, F value) {
+    const int tid = threadIdx.x;
+    float* wk = reinterpret_cast<float*>(c.smem + WORK_OFF);
+    const int u0 = (int)((unsigned)a.N * (unsigned)c.cta / (unsigned)c.nctas);
+    const int u1 = (int)((unsigned)a.N * (unsigned)(c.cta + 1) / (unsigned)c.nctas);
+    float ssq_acc = 0.f;
+    a.epi = EPI_STORE;
+    if (tid < M_MAX) wk[LW_RS + tid] = 1.0f;
+    for (int sc0 = u0; sc0 < u1; sc0 += SC_ROWS) {
+        const int nu = min(SC_ROWS, u1 - sc0);
+        for (int idx = tid; idx < nu * a.M; idx += NTHREADS) {
+            const int r = idx % nu, m = idx / nu;
+            wk[LW_ACC + (size_t)r * MP + m] = value(m, sc0 + r);
+        }
+        cta_sync();
+        emit_rows(a, wk, sc0, nu, false, ssq_acc);
+        cta_sync();
+    }
+    if (a.ssq_out && tid < a.M) a.ssq_out[(size_t)tid * c.nctas + c.cta] = ssq_acc;
 }
 
 // Plain path for any storage type (fp32 models, odd shapes, and a cross-check of the tensor-core
@@ -742,19 +849,13 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
     cta_sync();
 }
 
-// Which path an operator takes; the producer and the consumers must agree.
-template <typename WT> __device__ __forceinline__ bool lin_streams(const LinArgs& a, bool force_simple);
-template <> __device__ __forceinline__ bool lin_streams<float>(const LinArgs&, bool) { return false; }
-template <> __device__ __forceinline__ bool lin_streams<__nv_bfloat16>(const LinArgs& a, bool force_simple) {
-    return !force_simple && (a.K & 15) == 0;
-}
-
-// One linear operator, called by every thread of the CTA.  Consumers return after their part;
-// whether the grid must stop is learnt at the next grid barrier.  The producer returns false when
-// one of its waits gave up.
+// One linear operator, called by every thread of the CTA; `stream` selects the streamed tensor-core
+// path (bf16 weights, every K a multiple of 16; decided once per model so that the packed activation
+// rows exist wherever they are read).  Consumers return after their part; whether the grid must stop
+// is learnt at the next grid barrier.  The producer returns false when one of its waits gave up.
 template <typename WT>
-__device__ __forceinline__ bool linear_op(const LinArgs& a, Ctx& c, bool force_simple) {
-    if (lin_streams<WT>(a, force_simple)) {
+__device__ __forceinline__ bool linear_op(const LinArgs& a, Ctx& c, bool stream) {
+    if (stream) {
         if (c.producer) return lin_produce(a, c);
         if (a.M <= 4) lin_consume<4>(a, c); else if (a.M <= 8) lin_consume<8>(a, c); else lin_consume<16>(a, c);
         return true;
@@ -780,6 +881,7 @@ struct AttArgs {
     int M, pos0;           // rows sit at positions pos0 .. pos0+M-1; row i sees keys 0 .. pos0+i
     void* kc; void* vc;    // this layer's cache: [n_pages][H][page_size][hd]
     float* out;            // [M][d]
+    unsigned char* opk;    // packed copy of out for the output projection (nullable); d * 4 bytes per row
 };
 
 // Consumer threads only.  One work item = (head, KV split).  Keys come from the paged cache; the
@@ -942,7 +1044,9 @@ __device__ __noinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c
                     den += ldcg_f(ml + q * 2 + 1) * w;
                     num += ldcg_f(D.att_po + (((size_t)i * H + hh) * S_CAP + q) * hd + e) * w;
                 }
-                a.out[(size_t)i * d + hh * hd + e] = num / den;
+                const float ov = num / den;
+                a.out[(size_t)i * d + hh * hd + e] = ov;
+                if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
             }
         }
     }

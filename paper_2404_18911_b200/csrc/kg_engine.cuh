@@ -26,6 +26,11 @@ struct Program {
 #define KG_SYNC(where) do { if (!sync(where)) return false; } while (0)
 #define KG_LIN(args) do { if (!linear(args)) return false; } while (0)
 
+// Rows handed from one operator to the next: fp32 rows (residual input, plain path), their packed copy
+// scaled by the reader's norm gain, and the per-CTA sums of squares the reader's RMSNorm needs.
+struct ActIn { const float* x; const unsigned char* pk; const float* ssq; };
+struct ActOut { float* x; PkOut pk[2]; float* ssq; };
+
 template <typename WT>
 struct Engine {
     const Dev& D;
@@ -35,70 +40,97 @@ struct Engine {
     __device__ Engine(const Dev& d, Ctx& cx, const Program& p) : D(d), c(cx), pg(p) {}
 
     // ---- leaf operations: what a thread does depends on its role -------------------------------
-    __device__ __forceinline__ bool linear(const LinArgs& a) { return linear_op<WT>(a, c, pg.force_simple != 0); }
+    __device__ __forceinline__ bool streamed() const { return D.dm.stream != 0 && pg.force_simple == 0; }
+    __device__ __forceinline__ bool linear(const LinArgs& a) { return linear_op<WT>(a, c, streamed()); }
     __device__ __forceinline__ bool sync(int where) { return c.producer ? true : grid_sync(c, where); }
     __device__ __forceinline__ void attention(const AttArgs& at) { if (!c.producer) attention_op<WT>(D, at, c); }
 
     __device__ size_t cache_layer_stride() const {
         return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
     }
+    __device__ __forceinline__ size_t ldpk() const { return (size_t)D.dm.d * 4; }
+    __device__ __forceinline__ ActIn act_h() const { return ActIn{D.h, D.hA_pk, D.ssq_hA}; }
+    // the residual stream as an output, packed for a reader whose norm gain is `gain`
+    __device__ __forceinline__ ActOut out_h(const float* gain) const {
+        ActOut o; o.x = D.h; o.pk[0] = PkOut{gain, D.hA_pk}; o.pk[1] = PkOut{nullptr, nullptr}; o.ssq = D.ssq_hA; return o;
+    }
+    // norm gain of whatever reads the output of layer i: the next layer, or the LM head after the last one
+    __device__ __forceinline__ const float* next_gain(int i) const { return i + 1 < D.dm.L ? D.layers[i + 1].g1 : D.g_final; }
 
-    // h[i] = E[token_i]
-    __device__ void embed_rows(const int* toks_global, int tok_single, int M, float* out) {
+    // h[i] = E[token_i]; packed for layer 0
+    __device__ void embed_rows(const int* toks_global, int tok_single, int M) {
         if (c.producer) return;
         const int d = D.dm.d;
         const WT* E = reinterpret_cast<const WT*>(D.embed);
-        for (int idx = c.cta * NTHREADS + threadIdx.x; idx < M * d; idx += c.nctas * NTHREADS) {
-            const int i = idx / d, e = idx % d;
-            const int tok = toks_global ? __ldcg(toks_global + i) : tok_single;
-            out[idx] = wt_to_float<WT>(E[(size_t)tok * d + e]);
+        if (!streamed()) {
+            for (int idx = c.cta * NTHREADS + threadIdx.x; idx < M * d; idx += c.nctas * NTHREADS) {
+                const int i = idx / d, e = idx % d;
+                const int tok = toks_global ? __ldcg(toks_global + i) : tok_single;
+                D.h[idx] = wt_to_float<WT>(E[(size_t)tok * d + e]);
+            }
+            return;
         }
+        LinArgs a{};
+        a.N = d; a.M = M; a.out = D.h; a.ldo = d;
+        a.pk[0] = PkOut{D.layers[0].g1, D.hA_pk}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_hA;
+        emit_plain_rows(a, c, [&](int m, int e) {
+            const int tok = toks_global ? __ldcg(toks_global + m) : tok_single;
+            return wt_to_float<WT>(E[(size_t)tok * d + e]);
+        });
     }
 
     // One decoder block on M rows at positions pos0.. (Section 3.1's M^b layers):
     //   h  = x + Wo Attn(RMSNorm(x; g1));   out = h + Wdown(SiLU(Wgate n) * Wup n), n = RMSNorm(h; g2)
-    __device__ bool run_layer(int li, int M, int pos0, const float* xin, float* out) {
+    __device__ bool run_layer(int li, int M, int pos0, const ActIn& in, const ActOut& out) {
         const Dims& dm = D.dm;
         const LayerW lw = D.layers[li];
         LinArgs a{};
         a.M = M; a.eps = dm.eps;
         // q, k, v
         a.W = lw.wqkv; a.W2 = nullptr; a.N = 3 * dm.d; a.K = dm.d;
-        a.x = xin; a.ldx = dm.d; a.gain = lw.g1; a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
+        a.x = in.x; a.ldx = dm.d; a.gain = lw.g1; a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
+        a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
         KG_LIN(a);
         KG_SYNC(10);
         AttArgs at;
         at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
         at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)li * cache_layer_stride();
         at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)li * cache_layer_stride();
-        at.out = D.attn;
+        at.out = D.attn; at.opk = streamed() ? D.attn_pk : nullptr;
         attention(at);
         KG_SYNC(11);
         // output projection + residual -> h
         a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
-        a.epi = EPI_RESID; a.resid = xin; a.ldr = dm.d; a.out = D.h; a.ldo = dm.d;
+        a.xpk = D.attn_pk; a.ssq_in = nullptr;
+        a.epi = EPI_RESID; a.resid = in.x; a.ldr = dm.d; a.out = D.h; a.ldo = dm.d;
+        a.pk[0] = PkOut{lw.g2, D.hB_pk}; a.pk[1] = PkOut{nullptr, nullptr}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_hB;
         KG_LIN(a);
         KG_SYNC(12);
         // SwiGLU
         a.W = lw.wgate; a.W2 = lw.wup; a.N = dm.F; a.K = dm.d; a.x = D.h; a.ldx = dm.d; a.gain = lw.g2;
-        a.epi = EPI_SWIGLU; a.out = D.act; a.ldo = dm.F;
+        a.xpk = D.hB_pk; a.ssq_in = D.ssq_hB;
+        a.epi = EPI_SWIGLU; a.resid = nullptr; a.out = D.act; a.ldo = dm.F;
+        a.pk[0] = PkOut{nullptr, D.act_pk}; a.ldpk_out = dm.F * 4; a.ssq_out = nullptr;
         KG_LIN(a);
         KG_SYNC(13);
         a.W = lw.wdown; a.W2 = nullptr; a.N = dm.d; a.K = dm.F; a.x = D.act; a.ldx = dm.F; a.gain = nullptr;
-        a.epi = EPI_RESID; a.resid = D.h; a.ldr = dm.d; a.out = out; a.ldo = dm.d;
+        a.xpk = D.act_pk; a.ldpk = dm.F * 4; a.ssq_in = nullptr;
+        a.epi = EPI_RESID; a.resid = D.h; a.ldr = dm.d; a.out = out.x; a.ldo = dm.d;
+        a.pk[0] = out.pk[0]; a.pk[1] = out.pk[1]; a.ldpk_out = (int)ldpk(); a.ssq_out = out.ssq;
         KG_LIN(a);
         KG_SYNC(14);
         return true;
     }
 
-    // Adapter A (Section 3.1, Table 2): a = f + W^A_o Attn(RMSNorm(f; g_in)) on rows f[M] at pos0..;
+    // Adapter A (Section 3.1, Table 2): a = f + W^A_o Attn(RMSNorm(f; g_in)) on the rows `in` at pos0..;
     // with want_out == false only the adapter's K/V are appended (prefill).
-    __device__ bool run_adapter(int M, int pos0, const float* f, bool want_out) {
+    __device__ bool run_adapter(int M, int pos0, const ActIn& in, bool want_out) {
         const Dims& dm = D.dm;
         const LayerW lw = D.layers[dm.L];
         LinArgs a{};
         a.M = M; a.eps = dm.eps;
-        a.W = lw.wqkv; a.N = 3 * dm.d; a.K = dm.d; a.x = f; a.ldx = dm.d; a.gain = lw.g1;
+        a.W = lw.wqkv; a.N = 3 * dm.d; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = lw.g1;
+        a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
         a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
         KG_LIN(a);
         KG_SYNC(20);
@@ -106,25 +138,28 @@ struct Engine {
         at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
         at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)dm.L * cache_layer_stride();
         at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)dm.L * cache_layer_stride();
-        at.out = D.attn;
+        at.out = D.attn; at.opk = streamed() ? D.attn_pk : nullptr;
         attention(at);
         KG_SYNC(21);
         if (!want_out) return true;
         a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
-        a.epi = EPI_RESID; a.resid = f; a.ldr = dm.d; a.out = D.abuf; a.ldo = dm.d;
+        a.xpk = D.attn_pk; a.ssq_in = nullptr;
+        a.epi = EPI_RESID; a.resid = in.x; a.ldr = dm.d; a.out = D.abuf; a.ldo = dm.d;
+        a.pk[0] = PkOut{lw.g2, D.abuf_pk}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_abuf;
         KG_LIN(a);
         KG_SYNC(22);
         return true;
     }
 
-    // Shared LM head on rows x[M] (norm gain `gain`), then the merged (token, p) per row: the same
+    // Shared LM head on the rows `in` (norm gain `gain`), then the merged (token, p) per row: the same
     // values in every thread of every CTA, the producer warp included (it receives them through
     // shared memory and an mbarrier, which also holds it back until the result exists).
-    __device__ bool run_head(const float* x, int M, const float* gain, float* dbg, int* toks, float* ps) {
+    __device__ bool run_head(const ActIn& in, int M, const float* gain, float* dbg, int* toks, float* ps) {
         const Dims& dm = D.dm;
         LinArgs a{};
         a.M = M; a.eps = dm.eps;
-        a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = x; a.ldx = dm.d; a.gain = gain;
+        a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = gain;
+        a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
         a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
         a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
         if (!linear(a)) return false;
@@ -163,13 +198,29 @@ struct Engine {
     }
     __device__ bool leader() const { return c.cta == 0 && threadIdx.x == 0; }
 
-    // early feature of token `tok` at position pos -> feat slot
+    // the early-feature slot `slot` as an input of the adapter / of the first deep layer
+    __device__ __forceinline__ ActIn feat_for_adapter(int slot) const {
+        return ActIn{D.feat + (size_t)slot * D.dm.d, D.featA_pk + (size_t)slot * ldpk(), D.ssq_feat + (size_t)slot * c.nctas};
+    }
+    __device__ __forceinline__ ActIn feat_for_deep(int slot) const {
+        return ActIn{D.feat + (size_t)slot * D.dm.d, D.featD_pk + (size_t)slot * ldpk(), D.ssq_feat + (size_t)slot * c.nctas};
+    }
+
+    // early feature of token `tok` at position pos -> feat slot (fp32 and packed for both of its readers)
     __device__ bool shallow_pass(int tok, int pos, int slot) {
         const Dims& dm = D.dm;
-        embed_rows(nullptr, tok, 1, D.h);
+        embed_rows(nullptr, tok, 1);
         KG_SYNC(1);
-        for (int i = 0; i < dm.l; ++i)
-            if (!run_layer(i, 1, pos, D.h, (i == dm.l - 1) ? D.feat + (size_t)slot * dm.d : D.h)) return false;
+        for (int i = 0; i < dm.l; ++i) {
+            ActOut o = out_h(next_gain(i));
+            if (i == dm.l - 1) {
+                o.x = D.feat + (size_t)slot * dm.d;
+                o.pk[0] = PkOut{D.layers[dm.L].g1, D.featA_pk + (size_t)slot * ldpk()};
+                o.pk[1] = PkOut{D.layers[dm.l].g1, D.featD_pk + (size_t)slot * ldpk()};
+                o.ssq = D.ssq_feat + (size_t)slot * c.nctas;
+            }
+            if (!run_layer(i, 1, pos, act_h(), o)) return false;
+        }
         return true;
     }
 
@@ -183,11 +234,10 @@ struct Engine {
             if (!shallow_pass(cur, P + n_d, 1 + n_d)) return false;                 // f[n_d]
             if (n_d == pg.gamma || stop_after_shallow) break;
             const int MA = P + n_d - len_A + 1;                                     // 1, or 2 when the adapter cache lags
-            const float* f = D.feat + (size_t)(1 + n_d - (MA - 1)) * dm.d;
-            if (!run_adapter(MA, len_A, f, true)) return false;
+            if (!run_adapter(MA, len_A, feat_for_adapter(1 + n_d - (MA - 1)), true)) return false;
             int tk[M_MAX]; float pp[M_MAX];
-            if (!run_head(D.abuf + (size_t)(MA - 1) * dm.d, 1, D.layers[dm.L].g2,
-                          D.dbg_draft + (size_t)n_steps * dm.V, tk, pp)) return false;
+            const ActIn hin{D.abuf + (size_t)(MA - 1) * dm.d, D.abuf_pk + (size_t)(MA - 1) * ldpk(), D.ssq_abuf + (size_t)(MA - 1) * c.nctas};
+            if (!run_head(hin, 1, D.layers[dm.L].g2, D.dbg_draft + (size_t)n_steps * dm.V, tk, pp)) return false;
             len_A += MA;
             dconf[n_steps] = pp[0];
             n_steps++;
@@ -211,17 +261,22 @@ struct Engine {
         const Dims& dm = D.dm;
         const int M = n_d + 1;
         for (int i = dm.l; i < dm.L; ++i)
-            if (!run_layer(i, M, P, (i == dm.l) ? D.feat + dm.d : D.h, D.h)) return false;
+            if (!run_layer(i, M, P, (i == dm.l) ? feat_for_deep(1) : act_h(), out_h(next_gain(i)))) return false;
         int t[M_MAX]; float pp[M_MAX];
-        if (!run_head(D.h, M, D.g_final, D.dbg_verify, t, pp)) return false;
+        if (!run_head(act_h(), M, D.g_final, D.dbg_verify, t, pp)) return false;
         int k = 0;
         while (k < n_d && dtok[k] == t[k]) ++k;
         const int newP = P + k + 1;
         if (len_A > newP) len_A = newP;
         if (len_A < newP && !c.producer) {
-            // the adapter has not seen f[k] (k == n_d): keep it as the feature of position newP-1
+            // the adapter has not seen f[k] (k == n_d): keep it as the feature of position newP-1 (slot 0)
+            const int gtid = c.cta * NTHREADS + threadIdx.x, gn = c.nctas * NTHREADS;
             const float* src = D.feat + (size_t)(1 + k) * dm.d;
-            for (int e = c.cta * NTHREADS + threadIdx.x; e < dm.d; e += c.nctas * NTHREADS) D.feat[e] = __ldcg(src + e);
+            for (int e = gtid; e < dm.d; e += gn) D.feat[e] = __ldcg(src + e);
+            const unsigned* psrc = reinterpret_cast<const unsigned*>(D.featA_pk + (size_t)(1 + k) * ldpk());
+            unsigned* pdst = reinterpret_cast<unsigned*>(D.featA_pk);
+            for (int e = gtid; e < dm.d; e += gn) pdst[e] = __ldcg(psrc + e);
+            for (int e = gtid; e < c.nctas; e += gn) D.ssq_feat[e] = __ldcg(D.ssq_feat + (size_t)(1 + k) * c.nctas + e);
         }
         if (leader()) {
             State* st = D.st;
@@ -246,13 +301,19 @@ struct Engine {
         tk[0] = 0;
         for (int c0 = 0; c0 < n; c0 += M_MAX) {
             const int M = min(M_MAX, n - c0);
-            embed_rows(D.prompt + c0, 0, M, D.h);
+            embed_rows(D.prompt + c0, 0, M);
             KG_SYNC(2);
-            for (int i = 0; i < dm.l; ++i) if (!run_layer(i, M, c0, D.h, D.h)) return false;
-            if (!run_adapter(M, c0, D.h, false)) return false;
-            for (int i = dm.l; i < dm.L; ++i) if (!run_layer(i, M, c0, D.h, D.h)) return false;
-            if (c0 + M == n)
-                if (!run_head(D.h + (size_t)(M - 1) * dm.d, 1, D.g_final, D.dbg_verify, tk, pp)) return false;
+            for (int i = 0; i < dm.l; ++i) {
+                ActOut o = out_h(next_gain(i));
+                if (i == dm.l - 1) o.pk[1] = PkOut{D.layers[dm.L].g1, D.featA_pk};    // the adapter reads the same rows
+                if (!run_layer(i, M, c0, act_h(), o)) return false;
+            }
+            if (!run_adapter(M, c0, ActIn{D.h, D.featA_pk, D.ssq_hA}, false)) return false;
+            for (int i = dm.l; i < dm.L; ++i) if (!run_layer(i, M, c0, act_h(), out_h(next_gain(i)))) return false;
+            if (c0 + M == n) {
+                const ActIn hin{D.h + (size_t)(M - 1) * dm.d, D.hA_pk + (size_t)(M - 1) * ldpk(), D.ssq_hA + (size_t)(M - 1) * c.nctas};
+                if (!run_head(hin, 1, D.g_final, D.dbg_verify, tk, pp)) return false;
+            }
         }
         if (leader()) {
             State* st = D.st;
@@ -266,10 +327,10 @@ struct Engine {
         const Dims& dm = D.dm;
         int tk[M_MAX]; float pp[M_MAX];
         while (total < pg.n) {
-            embed_rows(nullptr, x0, 1, D.h);
+            embed_rows(nullptr, x0, 1);
             KG_SYNC(3);
-            for (int i = 0; i < dm.L; ++i) if (!run_layer(i, 1, P, D.h, D.h)) return false;
-            if (!run_head(D.h, 1, D.g_final, D.dbg_verify, tk, pp)) return false;
+            for (int i = 0; i < dm.L; ++i) if (!run_layer(i, 1, P, act_h(), out_h(next_gain(i)))) return false;
+            if (!run_head(act_h(), 1, D.g_final, D.dbg_verify, tk, pp)) return false;
             if (leader()) {
                 D.out_tokens[total] = tk[0];
                 D.st->P = P + 1; D.st->x0 = tk[0]; D.st->total = total + 1; D.st->len_A = -1;
