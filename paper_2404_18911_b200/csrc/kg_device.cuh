@@ -34,7 +34,6 @@ constexpr int NTHREADS = 256;      // consumer threads per CTA
 constexpr int NWARPS = NTHREADS / 32;
 constexpr int BLOCK_THREADS = NTHREADS + 32;   // + the producer warp (warp index NWARPS)
 constexpr int S_CAP = 16;          // most KV splits per head
-constexpr int ATT_TK = 64;         // keys per attention tile
 constexpr int HD_MAX = 128;
 
 // weight ring: RING slots of ST_ROWS weight rows x ST_K k-elements (bf16); rows are padded by 16
@@ -136,8 +135,13 @@ struct Ctrl {
     int att_last;
     int head_tok[M_MAX];
     float head_p[M_MAX];
+    // operator arguments, written once per operator by one thread of each role and read by all of its threads
+    // (kept here rather than on the per-thread stack, which the small L1 left beside 227 KB of shared memory cannot hold)
+    alignas(16) unsigned char args_cons[256];
+    alignas(16) unsigned char args_prod[256];
+    alignas(16) unsigned char args_att[64];
 };
-static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+static_assert(sizeof(Ctrl) <= CTRL_BYTES - 16, "control block too large");
 
 struct Ctx {
     int cta, nctas;
@@ -594,23 +598,36 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
             const int p0 = ph * pl.plen, len = min(pl.plen, K - p0);
             const int nsteps = len / 16;
             // ---- B fragments of this warp's k slice, kept in registers for every row group of the phase
+            // (every load is issued before any is used: steps past the end of the phase and rows >= M re-read valid
+            // data and are zeroed afterwards)
             unsigned fr[NS][FR];
+            {
+                const int last = nsteps - 1 - warp * NS;         // last valid step of this warp (< 0: none)
+                const unsigned char* pbase = xlane + (size_t)(p0 / 16) * 64;
 #pragma unroll
-            for (int s = 0; s < NS; ++s) {
-#pragma unroll
-                for (int q = 0; q < FR; ++q) fr[s][q] = 0u;
-                if (warp * NS + s < nsteps) {
-                    const unsigned char* px = xlane + (size_t)(p0 / 16 + s) * 64;
+                for (int s = 0; s < NS; ++s) {
+                    const unsigned char* px = pbase + (size_t)max(min(s, last), -warp * NS) * 64;
                     if (V == 4) {
-                        if (xrow < M) { const uint2 v = __ldcg(reinterpret_cast<const uint2*>(px)); fr[s][0] = v.x; fr[s][1] = v.y; }
+                        const uint2 v = __ldcg(reinterpret_cast<const uint2*>(xrow < M ? px : px - (size_t)xrow * a.ldpk));
+                        fr[s][0] = v.x; fr[s][1] = v.y;
                     } else {
 #pragma unroll
                         for (int n = 0; n < NACC; ++n) {
-                            if (xrow + 8 * n < M) {
-                                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(px + (size_t)(8 * n) * a.ldpk));
-                                fr[s][4 * n + 0] = v.x; fr[s][4 * n + 1] = v.y; fr[s][4 * n + 2] = v.z; fr[s][4 * n + 3] = v.w;
-                            }
+                            const int row = xrow + 8 * n;
+                            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(row < M ? px + (size_t)(8 * n) * a.ldpk : px - (size_t)xrow * a.ldpk));
+                            fr[s][4 * n + 0] = v.x; fr[s][4 * n + 1] = v.y; fr[s][4 * n + 2] = v.z; fr[s][4 * n + 3] = v.w;
                         }
+                    }
+                }
+#pragma unroll
+                for (int s = 0; s < NS; ++s) {
+                    const bool sv = s <= last;
+                    if (V == 4) {
+                        if (!(sv && xrow < M)) { fr[s][0] = 0u; fr[s][1] = 0u; }
+                    } else {
+#pragma unroll
+                        for (int n = 0; n < NACC; ++n)
+                            if (!(sv && xrow + 8 * n < M)) { fr[s][4 * n + 0] = 0u; fr[s][4 * n + 1] = 0u; fr[s][4 * n + 2] = 0u; fr[s][4 * n + 3] = 0u; }
                     }
                 }
             }
@@ -855,12 +872,23 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
 // is learnt at the next grid barrier.  The producer returns false when one of its waits gave up.
 template <typename WT>
 __device__ __forceinline__ bool linear_op(const LinArgs& a, Ctx& c, bool stream) {
-    if (stream) {
-        if (c.producer) return lin_produce(a, c);
-        if (a.M <= 4) lin_consume<4>(a, c); else if (a.M <= 8) lin_consume<8>(a, c); else lin_consume<16>(a, c);
-        return true;
+    static_assert(sizeof(LinArgs) <= 256, "argument slot too small");
+    if (c.producer) {
+        if (!stream) return true;
+        LinArgs* sa = reinterpret_cast<LinArgs*>(c.ctl->args_prod);
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) *sa = a;
+        __syncwarp();
+        return lin_produce(*sa, c);
     }
-    if (!c.producer) lin_simple<WT>(a, c);
+    LinArgs* sa = reinterpret_cast<LinArgs*>(c.ctl->args_cons);
+    if (threadIdx.x == 0) *sa = a;
+    cta_sync();
+    if (stream) {
+        if (sa->M <= 4) lin_consume<4>(*sa, c); else if (sa->M <= 8) lin_consume<8>(*sa, c); else lin_consume<16>(*sa, c);
+    } else {
+        lin_simple<WT>(*sa, c);
+    }
     return true;
 }
 
@@ -884,40 +912,154 @@ struct AttArgs {
     unsigned char* opk;    // packed copy of out for the output projection (nullable); d * 4 bytes per row
 };
 
-// Consumer threads only.  One work item = (head, KV split).  Keys come from the paged cache; the
-// rows of this pass are rotated (RoPE), rounded to the cache's storage type and appended to the
-// cache by the item whose key range contains them, then read back like any other key.  Every split
-// writes a partial (max, sum, o); the last split of a head to arrive merges them in split order.
-template <typename WT>
-__device__ __noinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
+// Consumer threads only.  One work item = (head, KV split); the eight warps of the CTA cut the item's
+// key range into eight slices and run an online-softmax pass over their slice without any CTA
+// barrier: a lane owns hd/32 consecutive dimensions, so a key or value row is one coalesced load of
+// the warp, q . k is finished by a butterfly of shuffles, and o += p v stays in the lane.  Keys are
+// taken eight at a time (their loads are issued together).  The rows of this pass are rotated
+// (RoPE), rounded to the cache's storage type and appended to the cache by the item whose key range
+// contains them, then read back like any other key.  The warps' (max, sum, o) are merged through
+// shared memory; with more than one split every item writes a partial and the last split of a head
+// to arrive merges them in split order.
+template <typename WT, int DPL> struct AttLoad;          // raw bits of DPL consecutive elements, and their conversion
+template <> struct AttLoad<__nv_bfloat16, 4> {
+    typedef uint2 Raw;
+    static __device__ __forceinline__ Raw ld(const __nv_bfloat16* p) { return __ldcg(reinterpret_cast<const uint2*>(p)); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
+        v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
+    }
+};
+template <> struct AttLoad<__nv_bfloat16, 2> {
+    typedef unsigned Raw;
+    static __device__ __forceinline__ Raw ld(const __nv_bfloat16* p) { return __ldcg(reinterpret_cast<const unsigned*>(p)); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[2]) { v[0] = __uint_as_float(r << 16); v[1] = __uint_as_float(r & 0xffff0000u); }
+};
+template <> struct AttLoad<__nv_bfloat16, 1> {
+    typedef unsigned short Raw;
+    static __device__ __forceinline__ Raw ld(const __nv_bfloat16* p) { return __ldcg(reinterpret_cast<const unsigned short*>(p)); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[1]) { v[0] = __uint_as_float((unsigned)r << 16); }
+};
+template <> struct AttLoad<float, 4> {
+    typedef float4 Raw;
+    static __device__ __forceinline__ Raw ld(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[4]) { v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w; }
+};
+template <> struct AttLoad<float, 2> {
+    typedef float2 Raw;
+    static __device__ __forceinline__ Raw ld(const float* p) { return __ldcg(reinterpret_cast<const float2*>(p)); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[2]) { v[0] = r.x; v[1] = r.y; }
+};
+template <> struct AttLoad<float, 1> {
+    typedef float Raw;
+    static __device__ __forceinline__ Raw ld(const float* p) { return __ldcg(p); }
+    static __device__ __forceinline__ void cvt(const Raw& r, float (&v)[1]) { v[0] = r; }
+};
+
+constexpr int ATT_G = 8;           // keys per group
+constexpr int ATT_RB = 4;          // rows per block
+constexpr int ATT_MB_STRIDE = HD_MAX + 2;   // merge buffer row: o[hd], max, sum
+
+// One warp: rows i0 .. i0+nr-1 of the pass against keys [kb, ke) of head hh.
+template <typename WT, int DPL>
+__device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, int hh, int i0, int nr, int kb, int ke,
+                                               const float* qs, float (&mrow)[ATT_RB], float (&lrow)[ATT_RB], float (&o)[ATT_RB][DPL]) {
+    const int lane = threadIdx.x & 31;
+    const int H = D.dm.H, hd = D.dm.hd, ps = D.dm.page_size;
+    const WT* kc = reinterpret_cast<const WT*>(a.kc);
+    const WT* vc = reinterpret_cast<const WT*>(a.vc);
+    float q[ATT_RB][DPL];
+#pragma unroll
+    for (int r = 0; r < ATT_RB; ++r) {
+        mrow[r] = -INFINITY; lrow[r] = 0.f;
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) { o[r][e] = 0.f; q[r][e] = r < nr ? qs[(i0 + r) * HD_MAX + lane * DPL + e] : 0.f; }
+    }
+    for (int g0 = kb; g0 < ke; g0 += ATT_G) {
+        // every load of the group is issued before any is used (keys past the end re-read the last key and are masked)
+        int pg[ATT_G];
+#pragma unroll
+        for (int j = 0; j < ATT_G; ++j) pg[j] = __ldg(D.page_table + min(g0 + j, ke - 1) / ps);
+        typename AttLoad<WT, DPL>::Raw kr[ATT_G], vr[ATT_G];
+#pragma unroll
+        for (int j = 0; j < ATT_G; ++j) {
+            const int pos = min(g0 + j, ke - 1);
+            const size_t base = (((size_t)pg[j] * H + hh) * ps + pos % ps) * hd + lane * DPL;
+            kr[j] = AttLoad<WT, DPL>::ld(kc + base);
+            vr[j] = AttLoad<WT, DPL>::ld(vc + base);
+        }
+        float kv[ATT_G][DPL], vv[ATT_G][DPL];
+#pragma unroll
+        for (int j = 0; j < ATT_G; ++j) { AttLoad<WT, DPL>::cvt(kr[j], kv[j]); AttLoad<WT, DPL>::cvt(vr[j], vv[j]); }
+        float s[ATT_G][ATT_RB];
+#pragma unroll
+        for (int j = 0; j < ATT_G; ++j) {
+#pragma unroll
+            for (int r = 0; r < ATT_RB; ++r) {
+                float d = 0.f;
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) d = fmaf(q[r][e], kv[j][e], d);
+#pragma unroll
+                for (int ofs = 16; ofs > 0; ofs >>= 1) d += __shfl_xor_sync(0xffffffffu, d, ofs);
+                const int pos = g0 + j;
+                s[j][r] = (pos < ke && r < nr && pos <= a.pos0 + i0 + r) ? d : -INFINITY;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < ATT_RB; ++r) {
+            float mg = s[0][r];
+#pragma unroll
+            for (int j = 1; j < ATT_G; ++j) mg = fmaxf(mg, s[j][r]);
+            const float mn = fmaxf(mrow[r], mg);
+            if (mn != -INFINITY) {
+                const float cf = mrow[r] == -INFINITY ? 0.f : expf(mrow[r] - mn);
+                float ls = lrow[r] * cf;
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) o[r][e] *= cf;
+#pragma unroll
+                for (int j = 0; j < ATT_G; ++j) {
+                    const float p = s[j][r] == -INFINITY ? 0.f : expf(s[j][r] - mn);
+                    ls += p;
+#pragma unroll
+                    for (int e = 0; e < DPL; ++e) o[r][e] = fmaf(p, vv[j][e], o[r][e]);
+                }
+                lrow[r] = ls; mrow[r] = mn;
+            }
+        }
+    }
+}
+
+template <typename WT, int DPL>
+__device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx& c) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int H = D.dm.H, hd = D.dm.hd, d = D.dm.d, ps = D.dm.page_size;
     const int M = a.M, pos0 = a.pos0;
     const int T = pos0 + M;
     const int half = hd >> 1;
-    int S = min(min(S_CAP, max(1, (2 * c.nctas) / H)), (T + ATT_TK - 1) / ATT_TK);
+    // number of KV splits: the one that leaves the fewest keys on the busiest CTA
+    int S = 1;
+    {
+        long long best = -1;
+        for (int sc = 1; sc <= S_CAP; ++sc) {
+            const int chunk_ = (T + sc - 1) / sc;
+            if (sc > 1 && chunk_ < 32) break;
+            const int waves = (H * sc + c.nctas - 1) / c.nctas;
+            const long long cost = (long long)waves * (chunk_ + 48);      // + a fixed cost per item
+            if (best < 0 || cost < best) { best = cost; S = sc; }
+        }
+    }
     const int chunk = (T + S - 1) / S;
     const float sc = rsqrtf((float)hd);
     WT* kc = reinterpret_cast<WT*>(a.kc);
     WT* vc = reinterpret_cast<WT*>(a.vc);
 
     float* qs = reinterpret_cast<float*>(c.smem + WORK_OFF);       // [M_MAX][HD_MAX]
-    float* Ks = qs + M_MAX * HD_MAX;                               // [ATT_TK][hd+4]
-    float* Vs = Ks + ATT_TK * (HD_MAX + 4);                        // [ATT_TK][hd]
-    float* Ss = Vs + ATT_TK * HD_MAX;                              // [M_MAX][ATT_TK]
-    float* mrun = Ss + M_MAX * ATT_TK;                             // [M_MAX] running max
-    float* lrun = mrun + M_MAX;                                    // [M_MAX] running sum
-    float* corr = lrun + M_MAX;                                    // [M_MAX]
-    const int kstr = hd + 4;
-    const int rgs = NTHREADS / hd;                                 // row groups in the PV phase
-    const int e_pv = tid % hd, rg_pv = tid / hd;
-    constexpr int PV_R = 8;                                        // rows per thread in PV (rgs >= 2)
-    constexpr int SC_G = NTHREADS / ATT_TK;                        // row groups in the score phase
+    float* mb = qs + M_MAX * HD_MAX;                               // [NWARPS][ATT_RB][ATT_MB_STRIDE]
+    KG_PROBE(20);
 
     for (int item = c.cta; item < H * S; item += c.nctas) {
         const int hh = item / S, s = item % S;
         const int kb = s * chunk, ke = min(T, kb + chunk);
-        cta_sync();
         // q rows: RoPE, pre-scaled by 1/sqrt(hd)
         for (int idx = tid; idx < M * half; idx += NTHREADS) {
             const int i = idx / half, e = idx % half;
@@ -942,120 +1084,101 @@ __device__ __noinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c
                 vc[base + e + half] = float_to_wt<WT>(ldcg_f(src + 2 * d + e + half));
             }
         }
-        if (tid < M_MAX) { mrun[tid] = -INFINITY; lrun[tid] = 0.f; }
-        float o[PV_R];
-#pragma unroll
-        for (int r = 0; r < PV_R; ++r) o[r] = 0.f;
         cta_sync();
-
-        for (int tb = kb; tb < ke; tb += ATT_TK) {
-            const int nk = min(ATT_TK, ke - tb);
-            // stage K and V tiles as fp32
-            for (int idx = tid; idx < nk * (hd / 4); idx += NTHREADS) {
-                const int j = idx / (hd / 4), e4 = (idx % (hd / 4)) * 4;
-                const int pos = tb + j;
-                const size_t base = (((size_t)D.page_table[pos / ps] * H + hh) * ps + pos % ps) * hd + e4;
-                const float4 kv = load4_cg<WT>(kc + base), vv = load4_cg<WT>(vc + base);
-                *reinterpret_cast<float4*>(Ks + j * kstr + e4) = kv;
-                *reinterpret_cast<float4*>(Vs + j * hd + e4) = vv;
-            }
-            cta_sync();
-            // scores: thread (key j, row group rgq) -> rows i = rgq, rgq + SC_G, ...
-            {
-                const int j = tid % ATT_TK, rgq = tid / ATT_TK;
-                const int pos = tb + j;
-                for (int i = rgq; i < M; i += SC_G) {
-                    float s0 = 0.f;
-                    if (j < nk) {
-                        const float* kr = Ks + j * kstr;
-                        const float* q0 = qs + i * HD_MAX;
-                        for (int e4 = 0; e4 < hd; e4 += 4) {
-                            const float4 kv = *reinterpret_cast<const float4*>(kr + e4);
-                            const float4 a0 = *reinterpret_cast<const float4*>(q0 + e4);
-                            s0 = fmaf(kv.x, a0.x, fmaf(kv.y, a0.y, fmaf(kv.z, a0.z, fmaf(kv.w, a0.w, s0))));
-                        }
-                    }
-                    Ss[i * ATT_TK + j] = (j < nk && pos <= pos0 + i) ? s0 : -INFINITY;
-                }
-            }
-            cta_sync();
-            // online softmax bookkeeping: warp i owns rows i, i + NWARPS
-            for (int i = warp; i < M; i += NWARPS) {
-                const float v0 = Ss[i * ATT_TK + lane], v1 = Ss[i * ATT_TK + lane + 32];
-                const float mo = mrun[i];
-                const float mn = fmaxf(mo, warp_max(fmaxf(v0, v1)));
-                float p0 = 0.f, p1 = 0.f, cf = 1.f;
-                if (mn != -INFINITY) {
-                    p0 = expf(v0 - mn); p1 = expf(v1 - mn);
-                    cf = (mo == -INFINITY) ? 0.f : expf(mo - mn);
-                }
-                Ss[i * ATT_TK + lane] = p0; Ss[i * ATT_TK + lane + 32] = p1;
-                const float ps_ = warp_sum(p0 + p1);
-                if (lane == 0) { lrun[i] = lrun[i] * cf + ps_; mrun[i] = mn; corr[i] = cf; }
-            }
-            cta_sync();
-            // o += P V : thread (element e, row group) -> rows i = rg_pv + rgs * r
-            if (rg_pv < rgs) {
+        KG_PROBE(21);
+        // this warp's slice of the item's keys, in whole groups
+        const int nkeys = ke - kb;
+        const int per = ((nkeys + NWARPS - 1) / NWARPS + ATT_G - 1) / ATT_G * ATT_G;
+        const int wb = min(ke, kb + warp * per), we = min(ke, wb + per);
+        for (int i0 = 0; i0 < M; i0 += ATT_RB) {
+            const int nr = min(ATT_RB, M - i0);
+            float mrow[ATT_RB], lrow[ATT_RB], o[ATT_RB][DPL];
+            att_warp_slice<WT, DPL>(D, a, hh, i0, nr, wb, we, qs, mrow, lrow, o);
+            KG_PROBE(22);
 #pragma unroll
-                for (int r = 0; r < PV_R; ++r) {
-                    const int i = rg_pv + rgs * r;
-                    if (i < M) {
-                        float accv = o[r] * corr[i];
-                        const float* pr = Ss + i * ATT_TK;
-                        for (int j = 0; j < nk; ++j) accv = fmaf(pr[j], Vs[j * hd + e_pv], accv);
-                        o[r] = accv;
-                    }
-                }
+            for (int r = 0; r < ATT_RB; ++r) {
+                float* row = mb + ((size_t)warp * ATT_RB + r) * ATT_MB_STRIDE;
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) row[lane * DPL + e] = o[r][e];
+                if (lane == 0) { row[HD_MAX] = mrow[r]; row[HD_MAX + 1] = lrow[r]; }
             }
             cta_sync();
-        }
-        // partials
-        if (rg_pv < rgs) {
-#pragma unroll
-            for (int r = 0; r < PV_R; ++r) {
-                const int i = rg_pv + rgs * r;
-                if (i < M) D.att_po[(((size_t)i * H + hh) * S_CAP + s) * hd + e_pv] = o[r];
-            }
-        }
-        if (tid < M) {
-            D.att_ml[(((size_t)tid * H + hh) * S_CAP + s) * 2 + 0] = mrun[tid];
-            D.att_ml[(((size_t)tid * H + hh) * S_CAP + s) * 2 + 1] = lrun[tid];
-        }
-        __threadfence();
-        cta_sync();
-        if (tid == 0) {
-            const unsigned prev = atomicAdd(D.att_cnt + hh, 1u);
-            const int last = (prev == (unsigned)(S - 1));
-            c.ctl->att_last = last;
-            if (last) { D.att_cnt[hh] = 0u; __threadfence(); }
-        }
-        cta_sync();
-        if (*(volatile int*)&c.ctl->att_last) {
-            for (int idx = tid; idx < M * hd; idx += NTHREADS) {
-                const int i = idx / hd, e = idx % hd;
-                const float* ml = D.att_ml + ((size_t)i * H + hh) * S_CAP * 2;
+            for (int idx = tid; idx < nr * hd; idx += NTHREADS) {
+                const int r = idx / hd, e = idx % hd, i = i0 + r;
                 float mx = -INFINITY;
-                for (int q = 0; q < S; ++q) mx = fmaxf(mx, ldcg_f(ml + q * 2));
+#pragma unroll
+                for (int w = 0; w < NWARPS; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
                 float den = 0.f, num = 0.f;
-                for (int q = 0; q < S; ++q) {
-                    const float mq = ldcg_f(ml + q * 2);
-                    if (mq == -INFINITY) continue;
-                    const float w = expf(mq - mx);
-                    den += ldcg_f(ml + q * 2 + 1) * w;
-                    num += ldcg_f(D.att_po + (((size_t)i * H + hh) * S_CAP + q) * hd + e) * w;
+#pragma unroll
+                for (int w = 0; w < NWARPS; ++w) {
+                    const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
+                    const float mw = row[HD_MAX];
+                    if (mw != -INFINITY) {
+                        const float wgt = expf(mw - mx);
+                        den += row[HD_MAX + 1] * wgt;
+                        num += row[e] * wgt;
+                    }
                 }
-                const float ov = num / den;
-                a.out[(size_t)i * d + hh * hd + e] = ov;
-                if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
+                if (S == 1) {
+                    const float ov = num / den;
+                    a.out[(size_t)i * d + hh * hd + e] = ov;
+                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
+                } else {
+                    D.att_po[(((size_t)i * H + hh) * S_CAP + s) * hd + e] = num;
+                    if (e == 0) {
+                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 0] = mx;
+                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 1] = den;
+                    }
+                }
             }
+            cta_sync();
+            KG_PROBE(23);
+        }
+        if (S > 1) {
+            __threadfence();
+            cta_sync();
+            if (tid == 0) {
+                const unsigned prev = atomicAdd(D.att_cnt + hh, 1u);
+                const int last = (prev == (unsigned)(S - 1));
+                c.ctl->att_last = last;
+                if (last) { D.att_cnt[hh] = 0u; __threadfence(); }
+            }
+            cta_sync();
+            if (*(volatile int*)&c.ctl->att_last) {
+                for (int idx = tid; idx < M * hd; idx += NTHREADS) {
+                    const int i = idx / hd, e = idx % hd;
+                    const float* ml = D.att_ml + ((size_t)i * H + hh) * S_CAP * 2;
+                    float mx = -INFINITY;
+                    for (int q = 0; q < S; ++q) mx = fmaxf(mx, ldcg_f(ml + q * 2));
+                    float den = 0.f, num = 0.f;
+                    for (int q = 0; q < S; ++q) {
+                        const float mq = ldcg_f(ml + q * 2);
+                        if (mq == -INFINITY) continue;
+                        const float w = expf(mq - mx);
+                        den += ldcg_f(ml + q * 2 + 1) * w;
+                        num += ldcg_f(D.att_po + (((size_t)i * H + hh) * S_CAP + q) * hd + e) * w;
+                    }
+                    const float ov = num / den;
+                    a.out[(size_t)i * d + hh * hd + e] = ov;
+                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
+                }
+            }
+            cta_sync();
         }
     }
-    cta_sync();
 }
 
-static_assert((M_MAX * HD_MAX + ATT_TK * (HD_MAX + 4) + ATT_TK * HD_MAX + M_MAX * ATT_TK + 3 * M_MAX) * 4 <= WORK_BYTES,
-              "attention tiles do not fit in the work area");
-static_assert(9 * (LinGeom<8>::PLEN * 4 + 32) + (2 * NWARPS * 128 + SC_ROWS * MP + NWARPS * M_MAX + M_MAX) * 4 <= WORK_BYTES, "linear work area too large (M <= 8)");
-static_assert(17 * (LinGeom<16>::PLEN * 4 + 32) + (2 * NWARPS * 128 + SC_ROWS * MP + NWARPS * M_MAX + M_MAX) * 4 <= WORK_BYTES, "linear work area too large (M <= 16)");
+template <typename WT>
+__device__ __forceinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
+    static_assert(sizeof(AttArgs) <= 64, "argument slot too small");
+    AttArgs* sa = reinterpret_cast<AttArgs*>(c.ctl->args_att);
+    if (threadIdx.x == 0) *sa = a;
+    cta_sync();
+    if (D.dm.hd == 128) attention_impl<WT, 4>(D, *sa, c);
+    else if (D.dm.hd == 64) attention_impl<WT, 2>(D, *sa, c);
+    else attention_impl<WT, 1>(D, *sa, c);
+}
+
+static_assert((M_MAX * HD_MAX + NWARPS * ATT_RB * ATT_MB_STRIDE) * 4 <= WORK_BYTES, "attention buffers do not fit in the work area");
 
 }  // namespace kg
