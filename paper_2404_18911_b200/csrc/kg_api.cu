@@ -902,6 +902,7 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
     Dev D;
     std::memset(&D, 0, sizeof(D));
     D.dm.H = H; D.dm.hd = hd; D.dm.d = H * hd; D.dm.page_size = page_size; D.dm.theta = theta;
+    D.dm.n_pages = (pos0 + M + page_size - 1) / page_size;       // entries of page_table this call may touch
     for (int i = 0; i < hd / 2; ++i) D.inv_freq[i] = std::pow((double)theta, -2.0 * (double)i / (double)hd);
     D.page_table = page_table;
     D.att_po = (float*)((char*)scratch + sc.off_po); D.att_ml = (float*)((char*)scratch + sc.off_ml);

@@ -960,14 +960,26 @@ constexpr int ATT_G = 8;           // keys per group
 constexpr int ATT_RB = 4;          // rows per block
 constexpr int ATT_MB_STRIDE = HD_MAX + 2;   // merge buffer row: o[hd], max, sum
 
-// One warp: rows i0 .. i0+nr-1 of the pass against keys [kb, ke) of head hh.
+__device__ __forceinline__ float ex2f(float x) {             // 2^x, one special-function instruction
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// One warp: rows i0 .. i0+nr-1 of the pass against keys [kb, ke) of head hh.  Scores are kept in the log2
+// domain (q is pre-scaled by log2(e) / sqrt(hd)), so every exponential is one ex2.  The loads of the next
+// key group are in flight while the current one is reduced; the butterflies of the 32 scores of a group are
+// written level by level so that their shuffles pipeline.
 template <typename WT, int DPL>
 __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, int hh, int i0, int nr, int kb, int ke,
                                                const float* qs, float (&mrow)[ATT_RB], float (&lrow)[ATT_RB], float (&o)[ATT_RB][DPL]) {
+    typedef typename AttLoad<WT, DPL>::Raw Raw;
     const int lane = threadIdx.x & 31;
     const int H = D.dm.H, hd = D.dm.hd, ps = D.dm.page_size;
+    const int pos0 = a.pos0;
     const WT* kc = reinterpret_cast<const WT*>(a.kc);
     const WT* vc = reinterpret_cast<const WT*>(a.vc);
+    const int* page_table = D.page_table;
     float q[ATT_RB][DPL];
 #pragma unroll
     for (int r = 0; r < ATT_RB; ++r) {
@@ -975,22 +987,30 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
 #pragma unroll
         for (int e = 0; e < DPL; ++e) { o[r][e] = 0.f; q[r][e] = r < nr ? qs[(i0 + r) * HD_MAX + lane * DPL + e] : 0.f; }
     }
-    for (int g0 = kb; g0 < ke; g0 += ATT_G) {
-        // every load of the group is issued before any is used (keys past the end re-read the last key and are masked)
-        int pg[ATT_G];
-#pragma unroll
-        for (int j = 0; j < ATT_G; ++j) pg[j] = __ldg(D.page_table + min(g0 + j, ke - 1) / ps);
-        typename AttLoad<WT, DPL>::Raw kr[ATT_G], vr[ATT_G];
+    if (kb >= ke) return;
+    // page table entries of a window of keys live in the lanes (lane p holds page first_page + p)
+    const int win = max(ATT_G, (31 * ps) / ATT_G * ATT_G);
+    int wstart = kb, first_page = kb / ps;
+    int pgs = __ldg(page_table + min(first_page + lane, D.dm.n_pages - 1));
+    Raw kr[ATT_G], vr[ATT_G];
+    auto issue = [&](int g0) {
+        if (g0 >= wstart + win) { wstart = g0; first_page = g0 / ps; pgs = __ldg(page_table + min(first_page + lane, D.dm.n_pages - 1)); }
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
             const int pos = min(g0 + j, ke - 1);
-            const size_t base = (((size_t)pg[j] * H + hh) * ps + pos % ps) * hd + lane * DPL;
+            const int pg = __shfl_sync(0xffffffffu, pgs, pos / ps - first_page);
+            const size_t base = (((size_t)pg * H + hh) * ps + pos % ps) * hd + lane * DPL;
             kr[j] = AttLoad<WT, DPL>::ld(kc + base);
             vr[j] = AttLoad<WT, DPL>::ld(vc + base);
         }
+    };
+    issue(kb);
+    for (int g0 = kb; g0 < ke; g0 += ATT_G) {
         float kv[ATT_G][DPL], vv[ATT_G][DPL];
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) { AttLoad<WT, DPL>::cvt(kr[j], kv[j]); AttLoad<WT, DPL>::cvt(vr[j], vv[j]); }
+        if (g0 + ATT_G < ke) issue(g0 + ATT_G);
+        KG_PROBE(25);
         float s[ATT_G][ATT_RB];
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
@@ -999,12 +1019,25 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
                 float d = 0.f;
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) d = fmaf(q[r][e], kv[j][e], d);
-#pragma unroll
-                for (int ofs = 16; ofs > 0; ofs >>= 1) d += __shfl_xor_sync(0xffffffffu, d, ofs);
-                const int pos = g0 + j;
-                s[j][r] = (pos < ke && r < nr && pos <= a.pos0 + i0 + r) ? d : -INFINITY;
+                s[j][r] = d;
             }
         }
+#pragma unroll
+        for (int ofs = 16; ofs > 0; ofs >>= 1) {
+#pragma unroll
+            for (int j = 0; j < ATT_G; ++j) {
+#pragma unroll
+                for (int r = 0; r < ATT_RB; ++r) s[j][r] += __shfl_xor_sync(0xffffffffu, s[j][r], ofs);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < ATT_G; ++j) {
+            const int pos = g0 + j;
+#pragma unroll
+            for (int r = 0; r < ATT_RB; ++r)
+                if (!(pos < ke && r < nr && pos <= pos0 + i0 + r)) s[j][r] = -INFINITY;
+        }
+        KG_PROBE(26);
 #pragma unroll
         for (int r = 0; r < ATT_RB; ++r) {
             float mg = s[0][r];
@@ -1012,13 +1045,13 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
             for (int j = 1; j < ATT_G; ++j) mg = fmaxf(mg, s[j][r]);
             const float mn = fmaxf(mrow[r], mg);
             if (mn != -INFINITY) {
-                const float cf = mrow[r] == -INFINITY ? 0.f : expf(mrow[r] - mn);
+                const float cf = ex2f(mrow[r] - mn);             // 0 when the running max was -inf
                 float ls = lrow[r] * cf;
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[r][e] *= cf;
 #pragma unroll
                 for (int j = 0; j < ATT_G; ++j) {
-                    const float p = s[j][r] == -INFINITY ? 0.f : expf(s[j][r] - mn);
+                    const float p = ex2f(s[j][r] - mn);          // 0 for masked keys
                     ls += p;
 #pragma unroll
                     for (int e = 0; e < DPL; ++e) o[r][e] = fmaf(p, vv[j][e], o[r][e]);
@@ -1049,7 +1082,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
         }
     }
     const int chunk = (T + S - 1) / S;
-    const float sc = rsqrtf((float)hd);
+    const float sc = rsqrtf((float)hd) * 1.4426950408889634f;      // 1/sqrt(hd), and log2(e): scores live in the log2 domain
     WT* kc = reinterpret_cast<WT*>(a.kc);
     WT* vc = reinterpret_cast<WT*>(a.vc);
 
@@ -1114,7 +1147,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                     const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
                     const float mw = row[HD_MAX];
                     if (mw != -INFINITY) {
-                        const float wgt = expf(mw - mx);
+                        const float wgt = ex2f(mw - mx);
                         den += row[HD_MAX + 1] * wgt;
                         num += row[e] * wgt;
                     }
@@ -1154,7 +1187,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                     for (int q = 0; q < S; ++q) {
                         const float mq = ldcg_f(ml + q * 2);
                         if (mq == -INFINITY) continue;
-                        const float w = expf(mq - mx);
+                        const float w = ex2f(mq - mx);
                         den += ldcg_f(ml + q * 2 + 1) * w;
                         num += ldcg_f(D.att_po + (((size_t)i * H + hh) * S_CAP + q) * hd + e) * w;
                     }
