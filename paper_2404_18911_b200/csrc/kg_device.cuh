@@ -38,7 +38,7 @@ constexpr int HD_MAX = 128;
 
 // weight ring: RING slots of ST_ROWS weight rows x ST_K k-elements (bf16); rows are padded by 16
 // bytes so that the eight row addresses of an ldmatrix fall into distinct bank groups
-constexpr int RING = 4;
+constexpr int RING = 6;
 constexpr int ST_ROWS = 8;
 constexpr int ST_K = 2048;
 constexpr int ST_ROW_BYTES = ST_K * 2 + 16;
@@ -49,7 +49,8 @@ constexpr int WORK_OFF = RING_OFF + RING * SLOT_BYTES;
 constexpr int SMEM_TOTAL = 232448;                      // 227 KB, the most one CTA may own
 constexpr int WORK_BYTES = SMEM_TOTAL - WORK_OFF;       // activations, reductions, attention tiles
 constexpr int SC_ROWS = 256;                            // rows whose accumulators live in shared memory at once
-constexpr int SIMPLE_XS_BYTES = WORK_BYTES - 4096;      // activation staging of the plain path
+// the plain path never runs beside the streamed one in a launch, so it stages its activations over the ring too
+constexpr int SIMPLE_XS_BYTES = SMEM_TOTAL - RING_OFF - 4096;
 
 constexpr int BAR_RELEASE = 32;                          // word index of the grid barrier's release word (its own 128-byte line)
 constexpr int BAR_BYTES = 256;
@@ -795,7 +796,7 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
     const WT* W = reinterpret_cast<const WT*>(a.W);
     const WT* W2 = reinterpret_cast<const WT*>(a.W2);
     const bool dual = W2 != nullptr;
-    char* work = c.smem + WORK_OFF;
+    char* work = c.smem + RING_OFF;
     float* xs = reinterpret_cast<float*>(work);                          // [M][K]
     float* rs = reinterpret_cast<float*>(work + SIMPLE_XS_BYTES);        // [M_MAX]
     float* wst = rs + M_MAX;                                             // [NWARPS][M_MAX][3] head stats
