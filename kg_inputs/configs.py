@@ -59,15 +59,15 @@ CONFIGS = {
                     n_prompt=32, n_gen=64, eta=0.6, gamma=6),
     "7b": KgShape("7b", 32, 4096, 32, 128, 11008, 32000, 2, "bf16",
                   logit_scale=8.0, max_seq=1024, page_size=16, gamma_max=10,
-                  deep_resid_scale=0.1, adapter_resid_scale=0.1,
+                  deep_resid_scale=0.03, adapter_resid_scale=0.03,      # measured: accept rate 0.65, CR 2.55, top-1 p 0.23..1.0
                   n_prompt=512, n_gen=256, eta=0.6, gamma=6),
     "13b": KgShape("13b", 40, 5120, 40, 128, 13824, 32000, 2, "bf16",
                    logit_scale=8.0, max_seq=2048 + 512 + 64, page_size=16, gamma_max=10,
-                   deep_resid_scale=0.1, adapter_resid_scale=0.1,
+                   deep_resid_scale=0.03, adapter_resid_scale=0.03,
                    n_prompt=2048, n_gen=512, eta=0.6, gamma=6),
     "33b": KgShape("33b", 60, 6656, 52, 128, 17920, 32000, 3, "bf16",
                    logit_scale=8.0, max_seq=4096 + 256 + 64, page_size=16, gamma_max=10,
-                   deep_resid_scale=0.1, adapter_resid_scale=0.1,
+                   deep_resid_scale=0.03, adapter_resid_scale=0.03,
                    n_prompt=4096, n_gen=256, eta=0.6, gamma=8),
 }
 
