@@ -120,6 +120,21 @@ class ClockSampler:
                 "samples": len(rows), "power_w_max": max(power) if power else None}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(units_per_rank_step, steps, world, ms_max):
+    """Whole-job throughput of `world` independent replicas: all units processed / the slowest rank's time."""
+    return world * units_per_rank_step * steps / (ms_max * 1e-3)
+
+
 # ------------------------------------------------------------------------------------ CPU oracle legs
 
 def _oracle_sample(shape_name, n_prompt_s, n_gen_s):
@@ -293,15 +308,12 @@ def run_kangaroo(args):
     sampler.stop()
     assert out_pin.tolist() == toks_dev, "kg_generate and prefill_device + decode disagree"
 
-    if dist is not None:
-        t = torch.tensor([ms_total, ms_e2e], device=f"cuda:{local_rank}", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, f"cuda:{local_rank}")
 
     if rank == 0:
         n_tok = shape.n_gen
-        value = world * n_tok * args.steps / (ms_total * 1e-3)
-        e2e = world * n_tok * args.steps / (ms_e2e * 1e-3)
+        value = job_throughput(n_tok, args.steps, world, ms_total)
+        e2e = job_throughput(n_tok, args.steps, world, ms_e2e)
         peak, peak_src = _measured_peaks()
         dec_bytes = traffic.decode_bytes(shape, st_log)
         dec_ms = statistics.mean(decode_ms)
