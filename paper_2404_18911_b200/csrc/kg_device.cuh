@@ -208,6 +208,8 @@ __device__ __forceinline__ bool mbar_wait(Ctx& c, unsigned long long* bar, unsig
     const long long t0 = clock64();
     unsigned spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        // the producer warp shares an issue port with two consumer warps: it backs off instead of spinning
+        if (c.producer) __nanosleep(200);
         if (((++spins) & 63u) == 0u) {
             if (*(volatile int*)&c.ctl->abort) return false;
             if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); return false; }
@@ -283,19 +285,15 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
     cta_sync();
     KG_PROBE(1);
     if (threadIdx.x == 0) {
-        // bar[0] counts arrivals (monotonic over the launch); bar[BAR_RELEASE] is written once per barrier
-        // by the last CTA to arrive, so the waiting CTAs poll a word nobody else is updating
+        // bar[0] counts arrivals (monotonic over the launch): one release-add, then poll until every CTA has arrived
         c.bar_target += (unsigned)c.nctas;
         const unsigned gen = c.bar_target;
-        __threadfence();
-        const unsigned prev = atomicAdd(c.bar, 1u);
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.bar) : "memory");
         int ok = 1;
-        if (prev + 1u == gen) {
-            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(c.bar + BAR_RELEASE), "r"(gen) : "memory");
-        } else {
+        {
             const long long t0 = clock64();
             unsigned spins = 0;
-            while ((int)(ld_acquire_u32(c.bar + BAR_RELEASE) - gen) < 0) {
+            while ((int)(ld_acquire_u32(c.bar) - gen) < 0) {
                 if (((++spins) & 63u) == 0u) {
                     if (*(volatile int*)&c.st->status != 0) { ok = 0; break; }
                     if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
