@@ -688,17 +688,32 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                 }
                 cta_sync();
                 {
-                    // element (weight row r16, activation row m) of the pair
-                    constexpr int NEL = V == 4 ? 64 : (V == 8 ? 128 : 256);
-                    if (tid < NEL) {
-                        const int r16 = V == 4 ? tid >> 2 : (V == 8 ? tid >> 3 : tid >> 4);
-                        const int m = V == 4 ? tid & 3 : (V == 8 ? tid & 7 : tid & 15);
-                        const float* rb = red + (size_t)(V == 16 ? 0 : buf) * NWARPS * 128 + (V == 16 ? (m >> 3) * 128 : 0) + r16 * 8 + (m & 7);
+                    // element (weight row r16, activation row m) of the pair; for M <= 8 every thread adds a share of the
+                    // eight k-slices and a fixed butterfly joins the shares, so that no warp lags behind the others
+                    if (V == 16) {
+                        const int r16 = tid >> 4, m = tid & 15;
+                        const float* rb = red + (m >> 3) * 128 + r16 * 8 + (m & 7);
                         float v = 0.f;
 #pragma unroll
-                        for (int w = 0; w < NWARPS; ++w) v += V == 4 ? rb[w * NACC * 128] + rb[w * NACC * 128 + 4] : rb[w * NACC * 128];
+                        for (int w = 0; w < NWARPS; ++w) v += rb[w * NACC * 128];
                         float* dst = acc_s + (size_t)((si >> 1) * 16 + r16) * MP + m;
                         *dst = ph == 0 ? v : *dst + v;
+                    } else {
+                        constexpr int TPE = V == 4 ? 4 : 2;                  // threads per element
+                        constexpr int WPT = NWARPS / TPE;                    // k-slices per thread
+                        const int e = tid / TPE, q = tid % TPE;
+                        const int r16 = V == 4 ? e >> 2 : e >> 3;
+                        const int m = V == 4 ? e & 3 : e & 7;
+                        const float* rb = red + (size_t)buf * NWARPS * 128 + r16 * 8 + m;
+                        float v = 0.f;
+#pragma unroll
+                        for (int w = 0; w < WPT; ++w) v += V == 4 ? rb[(q * WPT + w) * 128] + rb[(q * WPT + w) * 128 + 4] : rb[(q * WPT + w) * 128];
+#pragma unroll
+                        for (int o = 1; o < TPE; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (q == 0) {
+                            float* dst = acc_s + (size_t)((si >> 1) * 16 + r16) * MP + m;
+                            *dst = ph == 0 ? v : *dst + v;
+                        }
                     }
                 }
                 KG_PROBE(14);
