@@ -49,7 +49,7 @@ typedef struct {
     int32_t exit_layer;                      /* l, 1 <= l < L (Section 3.1) */
     int32_t dtype;                           /* KG_F32 | KG_BF16 */
     float rms_eps, rope_theta, logit_scale;  /* logits z = logit_scale * W_head y */
-    int32_t max_seq, page_size, gamma_max;   /* KV capacity in tokens; tokens per KV page; largest gamma */
+    int32_t max_seq, page_size, gamma_max;   /* KV capacity in tokens; tokens per KV page (a power of two); largest gamma */
     int32_t debug_logits;                    /* 1: keep every computed logit row in HBM for kg_debug_logits */
     int32_t page_shuffle;                    /* 1: non-identity page table (exercises the indirection) */
     /* synthetic initialisation, used when kg_init_model gets weights == NULL */

@@ -115,7 +115,7 @@ bool valid_config(const kg_config* c) {
     if (c->d_model % 8 || c->d_ffn % 8 || c->d_ffn <= 0 || c->vocab <= 1) return false;
     if (c->dtype != KG_F32 && c->dtype != KG_BF16) return false;
     if (c->gamma_max < 1 || c->gamma_max > KG_GAMMA_MAX) return false;
-    if (c->page_size < 1 || c->max_seq < 2) return false;
+    if (c->page_size < 1 || (c->page_size & (c->page_size - 1)) || c->max_seq < 2) return false;       // pages hold a power of two of tokens
     if (c->n_heads > 256) return false;
     if (c->vocab > (1 << 20) || c->d_ffn > (1 << 20)) return false;      // rows x CTAs must fit 32 bits
     // the plain path stages all rows of an operand in shared memory
@@ -327,6 +327,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     D.dm.V = cfg->vocab; D.dm.l = cfg->exit_layer; D.dm.eps = cfg->rms_eps; D.dm.theta = cfg->rope_theta;
     D.dm.logit_scale = cfg->logit_scale; D.dm.max_seq = cfg->max_seq; D.dm.page_size = cfg->page_size;
     D.dm.n_pages = (cfg->max_seq + cfg->page_size - 1) / cfg->page_size; D.dm.gamma_max = cfg->gamma_max;
+    for (D.dm.ps_shift = 0; (1 << D.dm.ps_shift) < cfg->page_size; ++D.dm.ps_shift) {}
     D.dm.debug = cfg->debug_logits;
     for (int i = 0; i < cfg->head_dim / 2; ++i)
         D.inv_freq[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
@@ -895,7 +896,8 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
                                float* out, void* scratch, void* stream) {
     if (!qkv || !kc || !vc || !page_table || !out || !scratch) return KG_E_ARG;
     if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
-    if (M < 1 || M > KG_M_MAX || pos0 < 0 || H < 1 || H > 256 || (hd != 32 && hd != 64 && hd != 128) || page_size < 1) return KG_E_ARG;
+    if (M < 1 || M > KG_M_MAX || pos0 < 0 || H < 1 || H > 256 || (hd != 32 && hd != 64 && hd != 128) || page_size < 1 ||
+        (page_size & (page_size - 1))) return KG_E_ARG;
     if ((size_t)H * hd > 8192) return KG_E_ARG;
     OpScratch sc = op_layout();
     cudaStream_t s = (cudaStream_t)stream;
@@ -903,6 +905,7 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
     std::memset(&D, 0, sizeof(D));
     D.dm.H = H; D.dm.hd = hd; D.dm.d = H * hd; D.dm.page_size = page_size; D.dm.theta = theta;
     D.dm.n_pages = (pos0 + M + page_size - 1) / page_size;       // entries of page_table this call may touch
+    for (D.dm.ps_shift = 0; (1 << D.dm.ps_shift) < page_size; ++D.dm.ps_shift) {}
     for (int i = 0; i < hd / 2; ++i) D.inv_freq[i] = std::pow((double)theta, -2.0 * (double)i / (double)hd);
     D.page_table = page_table;
     D.att_po = (float*)((char*)scratch + sc.off_po); D.att_ml = (float*)((char*)scratch + sc.off_ml);

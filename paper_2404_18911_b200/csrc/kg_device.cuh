@@ -68,6 +68,7 @@ struct Dims {
     int L, d, H, hd, F, V, l;
     float eps, theta, logit_scale;
     int max_seq, page_size, n_pages, gamma_max, debug;
+    int ps_shift;       // log2(page_size): page sizes are powers of two
     int stream;         // 1: linear operators take the streamed tensor-core path (bf16, d and F multiples of 16)
 };
 
@@ -982,14 +983,18 @@ __device__ __forceinline__ float ex2f(float x) {             // 2^x, one special
 
 // One warp: rows i0 .. i0+nr-1 of the pass against keys [kb, ke) of head hh.  Scores are kept in the log2
 // domain (q is pre-scaled by log2(e) / sqrt(hd)), so every exponential is one ex2.  The loads of the next
-// key group are in flight while the current one is reduced; the butterflies of the 32 scores of a group are
-// written level by level so that their shuffles pipeline.
+// key group are in flight while the current one is reduced.  A group's 8 x 4 partial dot products are summed
+// by a transposing butterfly (31 shuffles) that leaves score (key j, row r) in lane 4 j + r; that lane does the
+// online-softmax update of its row (lanes sharing r hold the same running max and sum), and the 32 probabilities
+// reach every lane through a few words of shared memory for o += p v.
 template <typename WT, int DPL>
 __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, int hh, int i0, int nr, int kb, int ke,
-                                               const float* qs, float (&mrow)[ATT_RB], float (&lrow)[ATT_RB], float (&o)[ATT_RB][DPL]) {
+                                               const float* qs, float* pbuf, float& m_lane, float& l_lane, float (&o)[ATT_RB][DPL]) {
     typedef typename AttLoad<WT, DPL>::Raw Raw;
+    static_assert(ATT_G == 8 && ATT_RB == 4, "the butterfly below is written for 8 keys x 4 rows");
     const int lane = threadIdx.x & 31;
-    const int H = D.dm.H, hd = D.dm.hd, ps = D.dm.page_size;
+    const int jl = lane >> 2, rl = lane & 3;
+    const int H = D.dm.H, hd = D.dm.hd, psh = D.dm.ps_shift, psm = D.dm.page_size - 1;
     const int pos0 = a.pos0;
     const WT* kc = reinterpret_cast<const WT*>(a.kc);
     const WT* vc = reinterpret_cast<const WT*>(a.vc);
@@ -997,23 +1002,23 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
     float q[ATT_RB][DPL];
 #pragma unroll
     for (int r = 0; r < ATT_RB; ++r) {
-        mrow[r] = -INFINITY; lrow[r] = 0.f;
 #pragma unroll
         for (int e = 0; e < DPL; ++e) { o[r][e] = 0.f; q[r][e] = r < nr ? qs[(i0 + r) * HD_MAX + lane * DPL + e] : 0.f; }
     }
+    m_lane = -INFINITY; l_lane = 0.f;
     if (kb >= ke) return;
     // page table entries of a window of keys live in the lanes (lane p holds page first_page + p)
-    const int win = max(ATT_G, (31 * ps) / ATT_G * ATT_G);
-    int wstart = kb, first_page = kb / ps;
+    const int win = max(ATT_G, ((31 << psh) >> 3) << 3);
+    int wstart = kb, first_page = kb >> psh;
     int pgs = __ldg(page_table + min(first_page + lane, D.dm.n_pages - 1));
     Raw kr[ATT_G], vr[ATT_G];
     auto issue = [&](int g0) {
-        if (g0 >= wstart + win) { wstart = g0; first_page = g0 / ps; pgs = __ldg(page_table + min(first_page + lane, D.dm.n_pages - 1)); }
+        if (g0 >= wstart + win) { wstart = g0; first_page = g0 >> psh; pgs = __ldg(page_table + min(first_page + lane, D.dm.n_pages - 1)); }
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
             const int pos = min(g0 + j, ke - 1);
-            const int pg = __shfl_sync(0xffffffffu, pgs, pos / ps - first_page);
-            const size_t base = (((size_t)pg * H + hh) * ps + pos % ps) * hd + lane * DPL;
+            const int pg = __shfl_sync(0xffffffffu, pgs, (pos >> psh) - first_page);
+            const size_t base = ((((size_t)pg * H + hh) << psh) + (pos & psm)) * hd + lane * DPL;
             kr[j] = AttLoad<WT, DPL>::ld(kc + base);
             vr[j] = AttLoad<WT, DPL>::ld(vc + base);
         }
@@ -1025,52 +1030,64 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
         for (int j = 0; j < ATT_G; ++j) { AttLoad<WT, DPL>::cvt(kr[j], kv[j]); AttLoad<WT, DPL>::cvt(vr[j], vv[j]); }
         if (g0 + ATT_G < ke) issue(g0 + ATT_G);
         KG_PROBE(25);
-        float s[ATT_G][ATT_RB];
+        float v[ATT_G * ATT_RB];
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
 #pragma unroll
             for (int r = 0; r < ATT_RB; ++r) {
-                float d = 0.f;
+                float dsum = 0.f;
 #pragma unroll
-                for (int e = 0; e < DPL; ++e) d = fmaf(q[r][e], kv[j][e], d);
-                s[j][r] = d;
+                for (int e = 0; e < DPL; ++e) dsum = fmaf(q[r][e], kv[j][e], dsum);
+                v[j * ATT_RB + r] = dsum;
             }
         }
+        // transposing butterfly: after the step with offset `ofs` a lane keeps the half of its values selected by that
+        // bit of its lane index, summed with the partner's; in the end lane L holds the full sum of value L
 #pragma unroll
         for (int ofs = 16; ofs > 0; ofs >>= 1) {
+            const bool up = (lane & ofs) != 0;
 #pragma unroll
-            for (int j = 0; j < ATT_G; ++j) {
-#pragma unroll
-                for (int r = 0; r < ATT_RB; ++r) s[j][r] += __shfl_xor_sync(0xffffffffu, s[j][r], ofs);
+            for (int i = 0; i < ofs; ++i) {
+                const float send = up ? v[i] : v[i + ofs];
+                const float keep = up ? v[i + ofs] : v[i];
+                v[i] = keep + __shfl_xor_sync(0xffffffffu, send, ofs);
             }
+        }
+        const int pos = g0 + jl;
+        float sv = (pos < ke && rl < nr && pos <= pos0 + i0 + rl) ? v[0] : -INFINITY;
+        float mg = sv;
+        mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, 4));
+        mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, 8));
+        mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, 16));
+        const float mn = fmaxf(m_lane, mg);
+        const float p = (sv == -INFINITY) ? 0.f : ex2f(sv - mn);
+        const float cf = (m_lane == -INFINITY) ? 0.f : ex2f(m_lane - mn);
+        float psum = p;
+        psum += __shfl_xor_sync(0xffffffffu, psum, 4);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 8);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 16);
+        l_lane = l_lane * cf + psum;
+        m_lane = mn;
+        KG_PROBE(26);
+        __syncwarp();
+        pbuf[lane] = p;
+        if (jl == 0) pbuf[32 + rl] = cf;
+        __syncwarp();
+        const float4 cfv = *reinterpret_cast<const float4*>(pbuf + 32);
+        const float cfa[4] = {cfv.x, cfv.y, cfv.z, cfv.w};
+#pragma unroll
+        for (int r = 0; r < ATT_RB; ++r) {
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) o[r][e] *= cfa[r];
         }
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
-            const int pos = g0 + j;
+            const float4 pj = *reinterpret_cast<const float4*>(pbuf + j * 4);
+            const float pa[4] = {pj.x, pj.y, pj.z, pj.w};
 #pragma unroll
-            for (int r = 0; r < ATT_RB; ++r)
-                if (!(pos < ke && r < nr && pos <= pos0 + i0 + r)) s[j][r] = -INFINITY;
-        }
-        KG_PROBE(26);
+            for (int r = 0; r < ATT_RB; ++r) {
 #pragma unroll
-        for (int r = 0; r < ATT_RB; ++r) {
-            float mg = s[0][r];
-#pragma unroll
-            for (int j = 1; j < ATT_G; ++j) mg = fmaxf(mg, s[j][r]);
-            const float mn = fmaxf(mrow[r], mg);
-            if (mn != -INFINITY) {
-                const float cf = ex2f(mrow[r] - mn);             // 0 when the running max was -inf
-                float ls = lrow[r] * cf;
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) o[r][e] *= cf;
-#pragma unroll
-                for (int j = 0; j < ATT_G; ++j) {
-                    const float p = ex2f(s[j][r] - mn);          // 0 for masked keys
-                    ls += p;
-#pragma unroll
-                    for (int e = 0; e < DPL; ++e) o[r][e] = fmaf(p, vv[j][e], o[r][e]);
-                }
-                lrow[r] = ls; mrow[r] = mn;
+                for (int e = 0; e < DPL; ++e) o[r][e] = fmaf(pa[r], vv[j][e], o[r][e]);
             }
         }
     }
@@ -1086,13 +1103,14 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
     // number of KV splits: the one that leaves the fewest keys on the busiest CTA
     int S = 1;
     {
-        long long best = -1;
+        const float inv_ctas = 1.0f / (float)c.nctas;
+        float best = -1.f;
+#pragma unroll
         for (int sc = 1; sc <= S_CAP; ++sc) {
-            const int chunk_ = (T + sc - 1) / sc;
-            if (sc > 1 && chunk_ < 32) break;
-            const int waves = (H * sc + c.nctas - 1) / c.nctas;
-            const long long cost = (long long)waves * (chunk_ + 48);      // + a fixed cost per item
-            if (best < 0 || cost < best) { best = cost; S = sc; }
+            const int chunk_ = (T + sc - 1) / sc;                                   // sc is a constant after unrolling
+            const float waves = ceilf((float)(H * sc) * inv_ctas - 1e-4f);
+            const float cost = waves * (float)(chunk_ + 48);                        // + a fixed cost per item
+            if ((sc == 1 || chunk_ >= 32) && (best < 0.f || cost < best)) { best = cost; S = sc; }
         }
     }
     const int chunk = (T + S - 1) / S;
@@ -1102,6 +1120,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
 
     float* qs = reinterpret_cast<float*>(c.smem + WORK_OFF);       // [M_MAX][HD_MAX]
     float* mb = qs + M_MAX * HD_MAX;                               // [NWARPS][ATT_RB][ATT_MB_STRIDE]
+    float* pbuf = mb + NWARPS * ATT_RB * ATT_MB_STRIDE + warp * 40;      // [NWARPS][40] probabilities of a key group
     KG_PROBE(20);
 
     for (int item = c.cta; item < H * S; item += c.nctas) {
@@ -1124,7 +1143,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                 float cs, sn; rope_cs(D, pos, e, cs, sn);
                 const float* src = a.qkv + (size_t)i * 3 * d + hh * hd;
                 const float k1 = ldcg_f(src + d + e), k2 = ldcg_f(src + d + e + half);
-                const size_t base = (((size_t)D.page_table[pos / ps] * H + hh) * ps + pos % ps) * hd;
+                const size_t base = (((size_t)D.page_table[pos >> D.dm.ps_shift] * H + hh) * ps + (pos & (ps - 1))) * hd;
                 kc[base + e] = float_to_wt<WT>(k1 * cs - k2 * sn);
                 kc[base + e + half] = float_to_wt<WT>(k2 * cs + k1 * sn);
                 vc[base + e] = float_to_wt<WT>(ldcg_f(src + 2 * d + e));
@@ -1139,15 +1158,15 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
         const int wb = min(ke, kb + warp * per), we = min(ke, wb + per);
         for (int i0 = 0; i0 < M; i0 += ATT_RB) {
             const int nr = min(ATT_RB, M - i0);
-            float mrow[ATT_RB], lrow[ATT_RB], o[ATT_RB][DPL];
-            att_warp_slice<WT, DPL>(D, a, hh, i0, nr, wb, we, qs, mrow, lrow, o);
+            float m_lane, l_lane, o[ATT_RB][DPL];
+            att_warp_slice<WT, DPL>(D, a, hh, i0, nr, wb, we, qs, pbuf, m_lane, l_lane, o);
             KG_PROBE(22);
 #pragma unroll
             for (int r = 0; r < ATT_RB; ++r) {
                 float* row = mb + ((size_t)warp * ATT_RB + r) * ATT_MB_STRIDE;
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) row[lane * DPL + e] = o[r][e];
-                if (lane == 0) { row[HD_MAX] = mrow[r]; row[HD_MAX + 1] = lrow[r]; }
+                if (lane == r) { row[HD_MAX] = m_lane; row[HD_MAX + 1] = l_lane; }       // lane r tracks row r
             }
             cta_sync();
             for (int idx = tid; idx < nr * hd; idx += NTHREADS) {
@@ -1226,6 +1245,6 @@ __device__ __forceinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx
     else attention_impl<WT, 1>(D, *sa, c);
 }
 
-static_assert((M_MAX * HD_MAX + NWARPS * ATT_RB * ATT_MB_STRIDE) * 4 <= WORK_BYTES, "attention buffers do not fit in the work area");
+static_assert((M_MAX * HD_MAX + NWARPS * ATT_RB * ATT_MB_STRIDE + NWARPS * 40) * 4 <= WORK_BYTES, "attention buffers do not fit in the work area");
 
 }  // namespace kg
