@@ -1,6 +1,8 @@
 """CUDA path vs CPU oracle through the C ABI: bit-exact tokens and accept lengths, logits within
 2e-2, confidences within 1e-3 (tolerances of the benchmark spec), on the tiny fp32 model, small
 bf16 models (tensor-core path, several tiles and ragged tails) and sampled rounds of the 7B shape."""
+import os
+
 import numpy as np
 import pytest
 
@@ -172,3 +174,52 @@ def test_api_errors(binding):
         g.draft(0.6, 6)
     assert e.value.status == b.KG_E_STATE                     # a draft is already pending
     g.verify()
+
+
+def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0):
+    """Full-size shape, short prompt: a handful of lock-step rounds against the fp32 oracle (the oracle's
+    weights for these shapes only fit in fp32, and a full-length prompt would take it hours)."""
+    from parity_harness import lockstep
+    shape = ki.get_config(name).with_(max_seq=n_prompt + n_new + 32)
+    g = binding.KangarooModel(shape, debug_logits=True)
+    o = ko.KangarooOracle(shape, ki.make_weights(shape), np.float64 if name == "7b" else np.float32)
+    prompt = ki.make_prompt(shape, n_prompt).tolist()
+    res = lockstep(g, o, prompt, n_new, shape.eta, shape.gamma, rounds_mode)
+    assert len(res["flips"]) <= 1, res["flips"]
+    assert res["max_logit_err"] < 2e-2 and res["max_conf_err"] < 1e-3, res
+    assert all(1 <= s <= shape.gamma + 1 for s in res["S"])
+    return res
+
+
+def test_7b_shape_sampled_rounds(binding):
+    """The benchmark's model (7B shape, bf16, l = 2) on a 24-token prompt: every round's drafts, confidences,
+    target tokens, accept lengths and logits against the oracle."""
+    res = _sampled_big_shape(binding, "7b", 24, 12)
+    assert len(res["tokens"]) >= 12
+
+
+@pytest.mark.skipif(os.environ.get("KG_BIG_PARITY") != "1", reason="the 13B oracle needs ~60 GB of host memory and minutes")
+def test_13b_shape_sampled_rounds(binding):
+    """As above for the 13B shape, against the fp32 oracle (its fp64 weights would not fit beside the fp32 ones)."""
+    _sampled_big_shape(binding, "13b", 16, 8)
+
+
+@pytest.mark.parametrize("name", ["13b", "33b"])
+def test_big_shapes_are_lossless_and_reproducible(binding, name):
+    """Properties that hold at any size, checked where the oracle is too slow: the self-speculative output equals
+    the same kernels' plain greedy decoding token for token (Section 3: acceptance is exact top-1 agreement), in both
+    stop modes, accept lengths lie in [1, gamma + 1], and a second run gives the same tokens bit for bit."""
+    shape = ki.get_config(name).with_(max_seq=192)
+    prompt = ki.make_prompt(shape, 40).tolist()
+    g = binding.KangarooModel(shape)
+    n = 48
+    toks, st = g.generate(prompt, n, shape.eta, shape.gamma, 0)
+    S = g.read_S()[: st["rounds"]]
+    assert all(1 <= s <= shape.gamma + 1 for s in S)
+    toks_drop, _ = g.generate(prompt, n, shape.eta, shape.gamma, 1)
+    assert toks_drop == toks
+    toks2, _ = g.generate(prompt, n, shape.eta, shape.gamma, 0)
+    assert toks2 == toks
+    g.reset()
+    g.prefill(prompt)
+    assert g.decode_ar(n) == toks
