@@ -24,7 +24,7 @@ def _resync(o, prompt, gpu_tokens):
     o.tokens[-1] = o.x0
 
 
-def lockstep(g, o, prompt, n_new, eta, gamma, mode, check_logits=True):
+def lockstep(g, o, prompt, n_new, eta, gamma, mode, check_logits=True, conf_tol=CONF_TOL):
     """g: binding.KangarooModel (debug_logits on when check_logits), o: KangarooOracle.
     Returns dict(tokens, S, flips, max_logit_err, max_conf_err)."""
     flips = []
@@ -63,19 +63,19 @@ def lockstep(g, o, prompt, n_new, eta, gamma, mode, check_logits=True):
                     raise Mismatch(f"draft logits step {j} differ by {err}")
             ce = abs(d["conf"][j] - r["conf"][j])
             max_ce = max(max_ce, ce)
-            if ce > CONF_TOL:
+            if ce > conf_tol:
                 raise Mismatch(f"confidence step {j}: {d['conf'][j]} vs {r['conf'][j]}")
             tg = d["tokens"][j] if j < len(d["tokens"]) else None
             to = r["drafts"][j] if j < len(r["drafts"]) else None
             if tg != to:
                 near_tie = ko.top2_gap(r["draft_logits"][j]) < LOGIT_TOL
-                near_eta = abs(r["conf"][j] - eta) < CONF_TOL
+                near_eta = abs(r["conf"][j] - eta) < conf_tol
                 if not (near_tie or near_eta):
                     raise Mismatch(f"draft token step {j}: {tg} vs {to}")
                 ok, why = False, ("draft", r["P"] + j)
                 break
         if ok and (d["n_steps"] != r["n_steps"] or d["n_drafted"] != r["n_drafted"]):
-            near_eta = any(abs(p - eta) < CONF_TOL for p in r["conf"])
+            near_eta = any(abs(p - eta) < conf_tol for p in r["conf"])
             if not near_eta:
                 raise Mismatch(f"draft counts differ: {d} vs n_d={r['n_drafted']} steps={r['n_steps']}")
             ok, why = False, ("eta", r["P"])

@@ -176,7 +176,7 @@ def test_api_errors(binding):
     g.verify()
 
 
-def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0):
+def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0, conf_tol=1e-3):
     """Full-size shape, short prompt: a handful of lock-step rounds against the fp32 oracle (the oracle's
     weights for these shapes only fit in fp32, and a full-length prompt would take it hours)."""
     from parity_harness import lockstep
@@ -184,9 +184,9 @@ def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0):
     g = binding.KangarooModel(shape, debug_logits=True)
     o = ko.KangarooOracle(shape, ki.make_weights(shape), np.float64 if name == "7b" else np.float32)
     prompt = ki.make_prompt(shape, n_prompt).tolist()
-    res = lockstep(g, o, prompt, n_new, shape.eta, shape.gamma, rounds_mode)
+    res = lockstep(g, o, prompt, n_new, shape.eta, shape.gamma, rounds_mode, conf_tol=conf_tol)
     assert len(res["flips"]) <= 1, res["flips"]
-    assert res["max_logit_err"] < 2e-2 and res["max_conf_err"] < 1e-3, res
+    assert res["max_logit_err"] < 2e-2 and res["max_conf_err"] < conf_tol, res
     assert all(1 <= s <= shape.gamma + 1 for s in res["S"])
     return res
 
@@ -196,12 +196,6 @@ def test_7b_shape_sampled_rounds(binding):
     target tokens, accept lengths and logits against the oracle."""
     res = _sampled_big_shape(binding, "7b", 24, 12)
     assert len(res["tokens"]) >= 12
-
-
-@pytest.mark.skipif(os.environ.get("KG_BIG_PARITY") != "1", reason="the 13B oracle needs ~60 GB of host memory and minutes")
-def test_13b_shape_sampled_rounds(binding):
-    """As above for the 13B shape, against the fp32 oracle (its fp64 weights would not fit beside the fp32 ones)."""
-    _sampled_big_shape(binding, "13b", 16, 8)
 
 
 @pytest.mark.parametrize("name", ["13b", "33b"])
