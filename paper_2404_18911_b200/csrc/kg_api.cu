@@ -761,7 +761,9 @@ __global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, 
     extern __shared__ __align__(128) char smem[];
     Ctx c;
     ctx_init(c, smem, nullptr, nullptr, false);
-    const bool ok = linear_op<WT>(a, c, stream != 0);
+    OpTable* t = reinterpret_cast<OpTable*>(c.producer ? c.ctl->tab_prod : c.ctl->tab_cons);
+    if (c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0) t->lin[0] = a;
+    const bool ok = linear_op<WT>(&t->lin[0], c, stream != 0, true);
     if (!ok && c.producer) ring_drain(c);
 }
 __global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* tok, float* p) {
@@ -772,7 +774,12 @@ __global__ void __launch_bounds__(BLOCK_THREADS, 1) op_attention_kernel(const __
     extern __shared__ __align__(128) char smem[];
     Ctx c;
     ctx_init(c, smem, nullptr, nullptr, false);
-    if (!c.producer) attention_op<WT>(D, a, c);
+    if (!c.producer) {
+        OpTable* t = reinterpret_cast<OpTable*>(c.ctl->tab_cons);
+        if (threadIdx.x == 0) t->att = a;
+        cta_sync();
+        attention_op<WT>(D, &t->att, c);
+    }
 }
 
 int g_force_simple_ops = 0;

@@ -43,7 +43,8 @@ constexpr int ST_ROWS = 8;
 constexpr int ST_K = 2048;
 constexpr int ST_ROW_BYTES = ST_K * 2 + 16;
 constexpr int SLOT_BYTES = ST_ROWS * ST_ROW_BYTES;
-constexpr int CTRL_BYTES = 1024;
+constexpr int CTRL_BYTES = 3072;
+constexpr int OP_TABLE_BYTES = 1024;                    // struct OpTable: the operator arguments of one layer
 constexpr int RING_OFF = CTRL_BYTES;
 constexpr int WORK_OFF = RING_OFF + RING * SLOT_BYTES;
 constexpr int SMEM_TOTAL = 232448;                      // 227 KB, the most one CTA may own
@@ -137,11 +138,11 @@ struct Ctrl {
     int att_last;
     int head_tok[M_MAX];
     float head_p[M_MAX];
-    // operator arguments, written once per operator by one thread of each role and read by all of its threads
-    // (kept here rather than on the per-thread stack, which the small L1 left beside 227 KB of shared memory cannot hold)
-    alignas(16) unsigned char args_cons[256];
-    alignas(16) unsigned char args_prod[256];
-    alignas(16) unsigned char args_att[64];
+    // operator arguments of a whole layer (struct OpTable), written once per layer by one thread of each role and
+    // read by all of its threads (kept here rather than on the per-thread stack, which the small L1 left beside
+    // 227 KB of shared memory cannot hold)
+    alignas(16) unsigned char tab_cons[OP_TABLE_BYTES];
+    alignas(16) unsigned char tab_prod[OP_TABLE_BYTES];
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES - 16, "control block too large");
 
@@ -427,6 +428,8 @@ __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
     const __nv_bfloat16* W = reinterpret_cast<const __nv_bfloat16*>(a.W);
     const __nv_bfloat16* W2 = reinterpret_cast<const __nv_bfloat16*>(a.W2);
     char* ring = c.smem + RING_OFF;
+    Ctrl* ctl = c.ctl;
+    int slot = c.slot; unsigned phase = c.phase; unsigned issued = c.issued;     // ring cursor, kept in registers here
     for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
         const int sc1 = min(pl.u1, sc0 + pl.sc_units);
         const int ngrp = (sc1 - sc0 + ST_ROWS - 1) / ST_ROWS;
@@ -438,18 +441,19 @@ __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
                 const int nvalid = min(ST_ROWS, sc1 - base);
                 const __nv_bfloat16* src = ((dual && (si & 1)) ? W2 : W) + (size_t)(base + lane) * a.K + p0;
                 int ok = 1;
-                if (lane == 0) ok = mbar_wait(c, &c.ctl->empty[c.slot], c.phase ^ 1u, 40) ? 1 : 0;
+                if (lane == 0) ok = mbar_wait(c, &ctl->empty[slot], phase ^ 1u, 40) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) return false;
-                if (lane == 0) mbar_arrive_expect_tx(&c.ctl->full[c.slot], (unsigned)(nvalid * len * 2));
+                if (!ok) { c.slot = slot; c.phase = phase; c.issued = issued; return false; }
+                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[slot], (unsigned)(nvalid * len * 2));
                 __syncwarp();
-                if (lane < nvalid) bulk_g2s(ring + (size_t)c.slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &c.ctl->full[c.slot]);
+                if (lane < nvalid) bulk_g2s(ring + (size_t)slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &ctl->full[slot]);
                 KG_PROBE(30);
-                c.issued++;
-                if (++c.slot == RING) { c.slot = 0; c.phase ^= 1u; }
+                issued++;
+                if (++slot == RING) { slot = 0; phase ^= 1u; }
             }
         }
     }
+    c.slot = slot; c.phase = phase; c.issued = issued;
     return true;
 }
 
@@ -557,6 +561,9 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
     float* acc_s = wk + LW_ACC;
     float* rs = wk + LW_RS;
     const char* ring = c.smem + RING_OFF;
+    Ctrl* ctl = c.ctl;
+    const int nctas = c.nctas, cta = c.cta;
+    int slot = c.slot; unsigned phase = c.phase;              // ring cursor, kept in registers here
 
     HeadStat hs[2];                                                        // EPI_HEAD: this warp tracks rows warp, warp + 8
     hs[0].zmax = hs[1].zmax = 0.f; hs[0].sum = hs[1].sum = 0.f; hs[0].arg = hs[1].arg = 0;
@@ -572,7 +579,7 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
         // thread (m, j) adds the partial sums of CTAs j, j + 16, ... of row m
         const int m = tid >> 4, j = tid & 15;
         float part = 0.f;
-        if (m < M) for (int q = j; q < c.nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * c.nctas + q);
+        if (m < M) for (int q = j; q < nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * nctas + q);
         wk[LW_RSP + tid] = part;
     }
     if (prefetched && a.epi != EPI_HEAD) {
@@ -636,14 +643,14 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
             const uint32_t a_lane = (uint32_t)((lane & 7) * ST_ROW_BYTES + (warp * NS * 16 + (lane >> 4) * 8) * 2);
             for (int si = 0; si < nst; si += 2) {
                 const bool two = si + 1 < nst;
-                const int slot_a = c.slot;
+                const int slot_a = slot;
                 const int slot_b = two ? (slot_a + 1 == RING ? 0 : slot_a + 1) : slot_a;
-                const unsigned phase_b = (two && slot_a + 1 == RING) ? c.phase ^ 1u : c.phase;
+                const unsigned phase_b = (two && slot_a + 1 == RING) ? phase ^ 1u : phase;
                 float acc[4][4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) { acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f; }
-                if (ok) ok = mbar_wait(c, &c.ctl->full[slot_a], c.phase, 41);
-                if (ok && two) ok = mbar_wait(c, &c.ctl->full[slot_b], phase_b, 41);
+                if (ok) ok = mbar_wait(c, &ctl->full[slot_a], phase, 41);
+                if (ok && two) ok = mbar_wait(c, &ctl->full[slot_b], phase_b, 41);
                 KG_PROBE(12);
                 if (ok) {
                     // ldmatrix x4: matrices 0, 2 = rows 0-7 (first stage), 1, 3 = rows 8-15 (second stage); k halves 0-7 | 8-15
@@ -669,9 +676,9 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                 }
                 __syncwarp();
                 KG_PROBE(13);
-                if (ok && lane == 0) { mbar_arrive(&c.ctl->empty[slot_a]); if (two) mbar_arrive(&c.ctl->empty[slot_b]); }
-                c.slot = slot_b; c.phase = phase_b;
-                if (++c.slot == RING) { c.slot = 0; c.phase ^= 1u; }
+                if (ok && lane == 0) { mbar_arrive(&ctl->empty[slot_a]); if (two) mbar_arrive(&ctl->empty[slot_b]); }
+                slot = slot_b; phase = phase_b;
+                if (++slot == RING) { slot = 0; phase ^= 1u; }
                 // ---- add the k-slices in warp order into the row accumulators
                 if (V == 16) cta_sync();                     // single partial-sum buffer: the previous pair's sums have been read
                 float* r = red + (size_t)(V == 16 ? 0 : buf) * NWARPS * 128 + (size_t)warp * NACC * 128;
@@ -770,10 +777,11 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int m = warp + q * NWARPS;
-            if (m < M) a.head_part[(size_t)c.cta * M_MAX + m] = make_float4(hs[q].zmax, hs[q].sum, __int_as_float(hs[q].arg), 0.f);
+            if (m < M) a.head_part[(size_t)cta * M_MAX + m] = make_float4(hs[q].zmax, hs[q].sum, __int_as_float(hs[q].arg), 0.f);
         }
     }
-    if (a.epi != EPI_HEAD && a.ssq_out && tid < M) a.ssq_out[(size_t)tid * c.nctas + c.cta] = ssq_acc;
+    if (a.epi != EPI_HEAD && a.ssq_out && tid < M) a.ssq_out[(size_t)tid * nctas + cta] = ssq_acc;
+    c.slot = slot; c.phase = phase;
 }
 
 // Rows that do not come out of a linear operator (token embeddings): every CTA takes its slice of
@@ -886,19 +894,14 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
 // rows exist wherever they are read).  Consumers return after their part; whether the grid must stop
 // is learnt at the next grid barrier.  The producer returns false when one of its waits gave up.
 template <typename WT>
-__device__ __forceinline__ bool linear_op(const LinArgs& a, Ctx& c, bool stream) {
-    static_assert(sizeof(LinArgs) <= 256, "argument slot too small");
+__device__ __forceinline__ bool linear_op(const LinArgs* sa, Ctx& c, bool stream, bool publish) {
+    // sa points into this role's operator table in shared memory; publish: the table was written just before
     if (c.producer) {
         if (!stream) return true;
-        LinArgs* sa = reinterpret_cast<LinArgs*>(c.ctl->args_prod);
-        __syncwarp();
-        if ((threadIdx.x & 31) == 0) *sa = a;
-        __syncwarp();
+        if (publish) __syncwarp();
         return lin_produce(*sa, c);
     }
-    LinArgs* sa = reinterpret_cast<LinArgs*>(c.ctl->args_cons);
-    if (threadIdx.x == 0) *sa = a;
-    cta_sync();
+    if (publish) cta_sync();
     if (stream) {
         if (sa->M <= 4) lin_consume<4>(*sa, c); else if (sa->M <= 8) lin_consume<8>(*sa, c); else lin_consume<16>(*sa, c);
     } else {
@@ -926,6 +929,10 @@ struct AttArgs {
     float* out;            // [M][d]
     unsigned char* opk;    // packed copy of out for the output projection (nullable); d * 4 bytes per row
 };
+
+// The operators of one layer (or of the adapter / the LM head), prepared together.
+struct OpTable { LinArgs lin[4]; AttArgs att; };
+static_assert(sizeof(OpTable) <= OP_TABLE_BYTES, "operator table too large");
 
 // Consumer threads only.  One work item = (head, KV split); the eight warps of the CTA cut the item's
 // key range into eight slices and run an online-softmax pass over their slice without any CTA
@@ -1235,11 +1242,8 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
 }
 
 template <typename WT>
-__device__ __forceinline__ void attention_op(const Dev& D, const AttArgs& a, Ctx& c) {
-    static_assert(sizeof(AttArgs) <= 64, "argument slot too small");
-    AttArgs* sa = reinterpret_cast<AttArgs*>(c.ctl->args_att);
-    if (threadIdx.x == 0) *sa = a;
-    cta_sync();
+__device__ __forceinline__ void attention_op(const Dev& D, const AttArgs* sa, Ctx& c) {
+    // sa points into the consumers' operator table in shared memory
     if (D.dm.hd == 128) attention_impl<WT, 4>(D, *sa, c);
     else if (D.dm.hd == 64) attention_impl<WT, 2>(D, *sa, c);
     else attention_impl<WT, 1>(D, *sa, c);

@@ -41,9 +41,15 @@ struct Engine {
 
     // ---- leaf operations: what a thread does depends on its role -------------------------------
     __device__ __forceinline__ bool streamed() const { return D.dm.stream != 0 && pg.force_simple == 0; }
-    __device__ __forceinline__ bool linear(const LinArgs& a) { return linear_op<WT>(a, c, streamed()); }
     __device__ __forceinline__ bool sync(int where) { return c.producer ? true : grid_sync(c, where); }
-    __device__ __forceinline__ void attention(const AttArgs& at) { if (!c.producer) attention_op<WT>(D, at, c); }
+    // this role's operator table in shared memory, and the one thread of the role that fills it
+    __device__ __forceinline__ OpTable* table() const {
+        if (c.producer) __syncwarp();        // the lanes have left the previous operator before lane 0 rewrites the table
+        return reinterpret_cast<OpTable*>(c.producer ? c.ctl->tab_prod : c.ctl->tab_cons);
+    }
+    __device__ __forceinline__ bool writer() const { return c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0; }
+    __device__ __forceinline__ bool linear(const LinArgs* a, bool publish) { return linear_op<WT>(a, c, streamed(), publish); }
+    __device__ __forceinline__ void attention(const AttArgs* at) { if (!c.producer) attention_op<WT>(D, at, c); }
 
     __device__ size_t cache_layer_stride() const {
         return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
@@ -79,45 +85,63 @@ struct Engine {
         });
     }
 
-    // One decoder block on M rows at positions pos0.. (Section 3.1's M^b layers):
-    //   h  = x + Wo Attn(RMSNorm(x; g1));   out = h + Wdown(SiLU(Wgate n) * Wup n), n = RMSNorm(h; g2)
-    __device__ bool run_layer(int li, int M, int pos0, const ActIn& in, const ActOut& out) {
+    // Arguments of the attention block of layer / adapter `li` on M rows at pos0: [0] q, k, v and [1] the output
+    // projection with its residual, plus the attention itself.
+    __device__ __forceinline__ void fill_attention_block(OpTable* t, const LayerW& lw, int li, int M, int pos0, const ActIn& in,
+                                                         float* o_out, const PkOut& o_pk, float* o_ssq) {
         const Dims& dm = D.dm;
-        const LayerW lw = D.layers[li];
-        LinArgs a{};
-        a.M = M; a.eps = dm.eps;
-        // q, k, v
-        a.W = lw.wqkv; a.W2 = nullptr; a.N = 3 * dm.d; a.K = dm.d;
-        a.x = in.x; a.ldx = dm.d; a.gain = lw.g1; a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
-        a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
-        KG_LIN(a);
-        KG_SYNC(10);
-        AttArgs at;
+        LinArgs& q = t->lin[0];
+        q = LinArgs{};
+        q.M = M; q.eps = dm.eps;
+        q.W = lw.wqkv; q.N = 3 * dm.d; q.K = dm.d;
+        q.x = in.x; q.ldx = dm.d; q.gain = lw.g1; q.xpk = in.pk; q.ldpk = (int)ldpk(); q.ssq_in = in.ssq;
+        q.epi = EPI_STORE; q.out = D.qkv; q.ldo = 3 * dm.d;
+        AttArgs& at = t->att;
         at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
         at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)li * cache_layer_stride();
         at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)li * cache_layer_stride();
         at.out = D.attn; at.opk = streamed() ? D.attn_pk : nullptr;
-        attention(at);
+        LinArgs& o = t->lin[1];
+        o = LinArgs{};
+        o.M = M; o.eps = dm.eps;
+        o.W = lw.wo; o.N = dm.d; o.K = dm.d; o.x = D.attn; o.ldx = dm.d;
+        o.xpk = D.attn_pk; o.ldpk = (int)ldpk();
+        o.epi = EPI_RESID; o.resid = in.x; o.ldr = dm.d; o.out = o_out; o.ldo = dm.d;
+        o.pk[0] = o_pk; o.ldpk_out = (int)ldpk(); o.ssq_out = o_ssq;
+    }
+
+    // One decoder block on M rows at positions pos0.. (Section 3.1's M^b layers):
+    //   h  = x + Wo Attn(RMSNorm(x; g1));   out = h + Wdown(SiLU(Wgate n) * Wup n), n = RMSNorm(h; g2)
+    __device__ bool run_layer(int li, int M, int pos0, const ActIn& in, const ActOut& out) {
+        const Dims& dm = D.dm;
+        OpTable* t = table();
+        if (writer()) {
+            const LayerW lw = D.layers[li];
+            fill_attention_block(t, lw, li, M, pos0, in, D.h, PkOut{lw.g2, D.hB_pk}, D.ssq_hB);
+            LinArgs& gu = t->lin[2];
+            gu = LinArgs{};
+            gu.M = M; gu.eps = dm.eps;
+            gu.W = lw.wgate; gu.W2 = lw.wup; gu.N = dm.F; gu.K = dm.d; gu.x = D.h; gu.ldx = dm.d; gu.gain = lw.g2;
+            gu.xpk = D.hB_pk; gu.ldpk = (int)ldpk(); gu.ssq_in = D.ssq_hB;
+            gu.epi = EPI_SWIGLU; gu.out = D.act; gu.ldo = dm.F;
+            gu.pk[0] = PkOut{nullptr, D.act_pk}; gu.ldpk_out = dm.F * 4;
+            LinArgs& dn = t->lin[3];
+            dn = LinArgs{};
+            dn.M = M; dn.eps = dm.eps;
+            dn.W = lw.wdown; dn.N = dm.d; dn.K = dm.F; dn.x = D.act; dn.ldx = dm.F;
+            dn.xpk = D.act_pk; dn.ldpk = dm.F * 4;
+            dn.epi = EPI_RESID; dn.resid = D.h; dn.ldr = dm.d; dn.out = out.x; dn.ldo = dm.d;
+            dn.pk[0] = out.pk[0]; dn.pk[1] = out.pk[1]; dn.ldpk_out = (int)ldpk(); dn.ssq_out = out.ssq;
+        }
+        if (!linear(&t->lin[0], true)) return false;
+        KG_SYNC(10);
+        attention(&t->att);
         KG_SYNC(11);
-        // output projection + residual -> h
-        a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
-        a.xpk = D.attn_pk; a.ssq_in = nullptr;
-        a.epi = EPI_RESID; a.resid = in.x; a.ldr = dm.d; a.out = D.h; a.ldo = dm.d;
-        a.pk[0] = PkOut{lw.g2, D.hB_pk}; a.pk[1] = PkOut{nullptr, nullptr}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_hB;
-        KG_LIN(a);
+        if (!linear(&t->lin[1], false)) return false;
         KG_SYNC(12);
-        // SwiGLU
-        a.W = lw.wgate; a.W2 = lw.wup; a.N = dm.F; a.K = dm.d; a.x = D.h; a.ldx = dm.d; a.gain = lw.g2;
-        a.xpk = D.hB_pk; a.ssq_in = D.ssq_hB;
-        a.epi = EPI_SWIGLU; a.resid = nullptr; a.out = D.act; a.ldo = dm.F;
-        a.pk[0] = PkOut{nullptr, D.act_pk}; a.ldpk_out = dm.F * 4; a.ssq_out = nullptr;
-        KG_LIN(a);
+        if (!linear(&t->lin[2], false)) return false;
         KG_SYNC(13);
-        a.W = lw.wdown; a.W2 = nullptr; a.N = dm.d; a.K = dm.F; a.x = D.act; a.ldx = dm.F; a.gain = nullptr;
-        a.xpk = D.act_pk; a.ldpk = dm.F * 4; a.ssq_in = nullptr;
-        a.epi = EPI_RESID; a.resid = D.h; a.ldr = dm.d; a.out = out.x; a.ldo = dm.d;
-        a.pk[0] = out.pk[0]; a.pk[1] = out.pk[1]; a.ldpk_out = (int)ldpk(); a.ssq_out = out.ssq;
-        KG_LIN(a);
+        if (!linear(&t->lin[3], false)) return false;
         KG_SYNC(14);
         return true;
     }
@@ -126,27 +150,17 @@ struct Engine {
     // with want_out == false only the adapter's K/V are appended (prefill).
     __device__ bool run_adapter(int M, int pos0, const ActIn& in, bool want_out) {
         const Dims& dm = D.dm;
-        const LayerW lw = D.layers[dm.L];
-        LinArgs a{};
-        a.M = M; a.eps = dm.eps;
-        a.W = lw.wqkv; a.N = 3 * dm.d; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = lw.g1;
-        a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
-        a.epi = EPI_STORE; a.out = D.qkv; a.ldo = 3 * dm.d;
-        KG_LIN(a);
+        OpTable* t = table();
+        if (writer()) {
+            const LayerW lw = D.layers[dm.L];
+            fill_attention_block(t, lw, dm.L, M, pos0, in, D.abuf, PkOut{lw.g2, D.abuf_pk}, D.ssq_abuf);
+        }
+        if (!linear(&t->lin[0], true)) return false;
         KG_SYNC(20);
-        AttArgs at;
-        at.qkv = D.qkv; at.M = M; at.pos0 = pos0;
-        at.kc = reinterpret_cast<WT*>(D.kcache) + (size_t)dm.L * cache_layer_stride();
-        at.vc = reinterpret_cast<WT*>(D.vcache) + (size_t)dm.L * cache_layer_stride();
-        at.out = D.attn; at.opk = streamed() ? D.attn_pk : nullptr;
-        attention(at);
+        attention(&t->att);
         KG_SYNC(21);
         if (!want_out) return true;
-        a.W = lw.wo; a.N = dm.d; a.K = dm.d; a.x = D.attn; a.ldx = dm.d; a.gain = nullptr;
-        a.xpk = D.attn_pk; a.ssq_in = nullptr;
-        a.epi = EPI_RESID; a.resid = in.x; a.ldr = dm.d; a.out = D.abuf; a.ldo = dm.d;
-        a.pk[0] = PkOut{lw.g2, D.abuf_pk}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_abuf;
-        KG_LIN(a);
+        if (!linear(&t->lin[1], false)) return false;
         KG_SYNC(22);
         return true;
     }
@@ -156,13 +170,17 @@ struct Engine {
     // shared memory and an mbarrier, which also holds it back until the result exists).
     __device__ bool run_head(const ActIn& in, int M, const float* gain, float* dbg, int* toks, float* ps) {
         const Dims& dm = D.dm;
-        LinArgs a{};
-        a.M = M; a.eps = dm.eps;
-        a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = gain;
-        a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
-        a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
-        a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
-        if (!linear(a)) return false;
+        OpTable* t = table();
+        if (writer()) {
+            LinArgs& a = t->lin[0];
+            a = LinArgs{};
+            a.M = M; a.eps = dm.eps;
+            a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = gain;
+            a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
+            a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
+            a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
+        }
+        if (!linear(&t->lin[0], true)) return false;
         if (c.producer) {
             // held back here until the consumers have the result
             int ok = 1;
