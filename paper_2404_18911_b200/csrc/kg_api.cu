@@ -759,8 +759,7 @@ OpScratch op_layout() {
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int stream) {
     extern __shared__ __align__(128) char smem[];
-    Ctx c;
-    ctx_init(c, smem, nullptr, nullptr, false);
+    Ctx& c = ctx_init(smem, nullptr, nullptr, false);
     OpTable* t = reinterpret_cast<OpTable*>(c.producer ? c.ctl->tab_prod : c.ctl->tab_cons);
     if (c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0) t->lin[0] = a;
     const bool ok = linear_op<WT>(&t->lin[0], c, stream != 0, true);
@@ -772,8 +771,7 @@ __global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* 
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) op_attention_kernel(const __grid_constant__ Dev D, AttArgs a) {
     extern __shared__ __align__(128) char smem[];
-    Ctx c;
-    ctx_init(c, smem, nullptr, nullptr, false);
+    Ctx& c = ctx_init(smem, nullptr, nullptr, false);
     if (!c.producer) {
         OpTable* t = reinterpret_cast<OpTable*>(c.ctl->tab_cons);
         if (threadIdx.x == 0) t->att = a;

@@ -143,9 +143,15 @@ struct Ctrl {
     // 227 KB of shared memory cannot hold)
     alignas(16) unsigned char tab_cons[OP_TABLE_BYTES];
     alignas(16) unsigned char tab_prod[OP_TABLE_BYTES];
+    // the per-role context (struct Ctx): one copy for the consumers, one for the producer warp
+    alignas(16) unsigned char ctx_cons[128];
+    alignas(16) unsigned char ctx_prod[128];
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES - 16, "control block too large");
 
+// State of one role (consumers / producer warp) of the CTA.  It lives in shared memory: every thread of the role
+// holds the same values, updates are the same in all of them, and between operators they are ordered by the
+// role's barriers; reading it never touches the per-thread stack.
 struct Ctx {
     int cta, nctas;
     unsigned bar_target;           // arrivals expected at the next grid barrier (thread 0 only)
@@ -262,20 +268,27 @@ __device__ __forceinline__ bool arg_better(float za, int ia, float zb, int ib) {
 }
 
 // ------------------------------------------------------------------------------------ CTA set-up
-// Called by every thread of the CTA at kernel start.
-__device__ __forceinline__ void ctx_init(Ctx& c, char* smem, State* st, unsigned* bar, bool grid) {
-    c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
-    c.ctl = reinterpret_cast<Ctrl*>(smem); c.grid = grid;
-    c.producer = threadIdx.x >= NTHREADS;
-    c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0;
+// Called by every thread of the CTA at kernel start; returns the context of the thread's role.
+__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, bool grid) {
+    static_assert(sizeof(Ctx) <= 128, "context slot too small");
+    Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
+    const bool producer = threadIdx.x >= NTHREADS;
+    Ctx& c = *reinterpret_cast<Ctx*>(producer ? ctl->ctx_prod : ctl->ctx_cons);
+    if (threadIdx.x == 0 || threadIdx.x == NTHREADS) {
+        c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
+        c.ctl = ctl; c.grid = grid;
+        c.producer = producer;
+        c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0;
+    }
     KG_PROBE_INIT();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < RING; ++i) { mbar_init(&c.ctl->full[i], 1); mbar_init(&c.ctl->empty[i], NWARPS); }
-        mbar_init(&c.ctl->mail, 1);
-        c.ctl->abort = 0; c.ctl->sync_ok = 1; c.ctl->att_last = 0;
+        for (int i = 0; i < RING; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], NWARPS); }
+        mbar_init(&ctl->mail, 1);
+        ctl->abort = 0; ctl->sync_ok = 1; ctl->att_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    return c;
 }
 
 // ------------------------------------------------------------------------------------ grid barrier

@@ -184,9 +184,11 @@ struct Engine {
         if (c.producer) {
             // held back here until the consumers have the result
             int ok = 1;
-            if ((threadIdx.x & 31) == 0) ok = mbar_wait(c, &c.ctl->mail, c.mail_phase, 42) ? 1 : 0;
+            const unsigned mp = c.mail_phase;
+            if ((threadIdx.x & 31) == 0) ok = mbar_wait(c, &c.ctl->mail, mp, 42) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            c.mail_phase ^= 1u;
+            if ((threadIdx.x & 31) == 0) c.mail_phase = mp ^ 1u;      // the context is shared by the warp: one lane updates it
+            __syncwarp();
             if (!ok) return false;
         } else {
             if (!grid_sync(c, 30)) return false;
@@ -384,8 +386,7 @@ struct Engine {
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
     extern __shared__ __align__(128) char smem[];
-    Ctx c;
-    ctx_init(c, smem, D.st, D.bar, true);
+    Ctx& c = ctx_init(smem, D.st, D.bar, true);
     Engine<WT> eng(D, c, pg);
     eng.run();
 }
