@@ -585,25 +585,29 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
     float ssq_acc = 0.f;
     KG_PROBE(10);
 
-    // ---- fetched now, used in the epilogue: the input rows' sums of squares, residual values, output gains
+    // ---- fetched early, used in the epilogue: the input rows' sums of squares, residual values, output gains.
+    // The requests go out right behind the first phase's fragment loads, which the first MMA waits for.
     const int nu0 = min(pl.u1 - pl.u0, pl.sc_units);
     const bool prefetched = nu0 <= PRE_NU;
-    if (a.ssq_in) {
-        // thread (m, j) adds the partial sums of CTAs j, j + 16, ... of row m
-        const int m = tid >> 4, j = tid & 15;
-        float part = 0.f;
-        if (m < M) for (int q = j; q < nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * nctas + q);
-        wk[LW_RSP + tid] = part;
-    }
-    if (prefetched && a.epi != EPI_HEAD) {
-        if (a.epi == EPI_RESID)
-            for (int i = tid; i < M * nu0; i += NTHREADS) cp_async4(wk + LW_PRES + (i / nu0) * PRE_NU + i % nu0, a.resid + (size_t)(i / nu0) * a.ldr + pl.u0 + i % nu0);
+    bool pre_pending = true;
+    auto epilogue_prefetch = [&]() {
+        if (a.ssq_in) {
+            // thread (m, j) adds the partial sums of CTAs j, j + 16, ... of row m
+            const int m = tid >> 4, j = tid & 15;
+            float part = 0.f;
+            if (m < M) for (int q = j; q < nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * nctas + q);
+            wk[LW_RSP + tid] = part;
+        }
+        if (prefetched && a.epi != EPI_HEAD) {
+            if (a.epi == EPI_RESID)
+                for (int i = tid; i < M * nu0; i += NTHREADS) cp_async4(wk + LW_PRES + (i / nu0) * PRE_NU + i % nu0, a.resid + (size_t)(i / nu0) * a.ldr + pl.u0 + i % nu0);
 #pragma unroll
-        for (int q = 0; q < 2; ++q)
-            if (a.pk[q].ptr && a.pk[q].gain)
-                for (int i = tid; i < nu0; i += NTHREADS) cp_async4(wk + LW_PREG + q * PRE_NU + i, a.pk[q].gain + pl.u0 + i);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
+            for (int q = 0; q < 2; ++q)
+                if (a.pk[q].ptr && a.pk[q].gain)
+                    for (int i = tid; i < nu0; i += NTHREADS) cp_async4(wk + LW_PREG + q * PRE_NU + i, a.pk[q].gain + pl.u0 + i);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
 
     // this lane's rows of the packed input: V = 4: row g & 3 (hi for g < 4, lo for g >= 4); else rows g (and g + 8)
     const int xrow = V == 4 ? (g & 3) : g;
@@ -639,6 +643,7 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                         }
                     }
                 }
+                if (pre_pending) { pre_pending = false; epilogue_prefetch(); }
 #pragma unroll
                 for (int s = 0; s < NS; ++s) {
                     const bool sv = s <= last;
