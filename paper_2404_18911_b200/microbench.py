@@ -117,13 +117,37 @@ def bench_ops(args, shape, torch, binding):
         del Ws, W2s
 
 
+def bench_sweep(args, shape, torch, binding):
+    """End-to-end decode of the workload for a grid of (eta, gamma): decode-only tokens/s (device time of the decode
+    launch), compression rate (Eq. 1), draft steps, and the speed-up over plain greedy decoding on the same kernels."""
+    import kg_inputs as ki
+    model = binding.KangarooModel(shape)
+    prompt = ki.make_prompt(shape).tolist()
+    n = shape.n_gen
+    # plain greedy baseline
+    model.reset(); model.prefill(prompt)
+    e0, e1 = _events(torch)
+    e0.record(); model.decode_ar(n, sync=False); e1.record(); torch.cuda.synchronize()
+    ar_ms = e0.elapsed_time(e1)
+    ref = model.read_tokens(n)
+    print(json.dumps({"point": "greedy", "tokens": n, "ms": ar_ms, "tokens_per_s": (n - 1) / ar_ms * 1e3}), flush=True)
+    for gamma in (2, 4, 6, 10):
+        for eta in (0.0, 0.2, 0.4, 0.6, 0.8):
+            toks, st = model.generate(prompt, n, eta, gamma)
+            assert toks == ref, "speculative output differs from greedy decoding"
+            print(json.dumps({"point": "kangaroo", "eta": eta, "gamma": gamma, "ms_decode": st["ms_decode"],
+                              "tokens_per_s": (n - 1) / st["ms_decode"] * 1e3, "speedup_vs_greedy": ar_ms / st["ms_decode"],
+                              "cr": st["cr"], "rounds": st["rounds"], "draft_steps": st["draft_steps"],
+                              "accept_rate": st["accepted"] / max(st["drafted"], 1)}), flush=True)
+
+
 def main():
     import torch
     import kg_inputs as ki
     from paper_2404_18911_b200 import binding, traffic, build_library
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="7b")
-    ap.add_argument("--what", default="steps", choices=["steps", "ops", "all"])
+    ap.add_argument("--what", default="steps", choices=["steps", "ops", "sweep", "all"])
     ap.add_argument("--T", default="128,512,2048,4096")
     ap.add_argument("--M", default="1,2,4,7,8")
     ap.add_argument("--reps", type=int, default=10)
@@ -135,6 +159,8 @@ def main():
         bench_steps(args, shape, torch, binding, traffic)
     if args.what in ("ops", "all"):
         bench_ops(args, shape, torch, binding)
+    if args.what == "sweep":
+        bench_sweep(args, shape, torch, binding)
     return 0
 
 
