@@ -31,6 +31,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the decode launch, from the ncu
+# capture summarised in profiles/kg_persistent_kernel_7b-4layers_decode.md (a 4-layer case of the same kernel; the
+# traffic is weights + KV and grows in proportion to the bytes a launch streams).  Set to None when the kernel changes.
+NCU_TRAFFIC_RATIO = 1.016
+
 METRIC = "batch-1 generated tokens/s"
 UNIT = "tokens/s"
 
@@ -333,7 +338,9 @@ def run_kangaroo(args):
             "roofline": {"bound": "hbm", "kernel": "kg_persistent_kernel (decode program: all rounds of one step)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8TBs": achieved / 8000.0, "peak_source": peak_src,
-                         "bytes_per_launch": dec_bytes, "ms_per_launch": dec_ms, "traffic": None},
+                         "bytes_per_launch": dec_bytes, "ms_per_launch": dec_ms,
+                         "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * dec_bytes),
+                         "traffic_source": "ncu dram bytes of a 4-layer launch of the same kernel, scaled by algorithmic bytes (x1.016)"},
             "breakdown": {"prefill_ms": statistics.mean(prefill_ms), "decode_ms": dec_ms,
                           "decode_only_tokens_per_s": (n_tok - 1) / (dec_ms * 1e-3),
                           "rounds": rounds, "cr": (n_tok - 1) / max(rounds, 1), "draft_steps": n_steps_total,
