@@ -1,6 +1,5 @@
 // Host side of the C ABI declared in include/kangaroo.h: arena layout, synthetic weight fill,
 // launches of the persistent decode kernel, small result copies.  No device allocation anywhere.
-#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -78,7 +77,7 @@ __global__ void pack_rows_kernel(const float* x, int ldx, int M, int K, const fl
         for (int k = k0 + threadIdx.x; k < k1; k += blockDim.x) {
             const float v = x[(size_t)m * ldx + k];
             ss += v * v;
-            pk_store(xpk + (size_t)m * ldpk, K, k, gain ? v * gain[k] : v);
+            pk_store(xpk + (size_t)m * ldpk, k, gain ? v * gain[k] : v);
         }
         ss = warp_sum(ss);
         if ((threadIdx.x & 31) == 0) sred[threadIdx.x >> 5] = ss;
@@ -103,7 +102,6 @@ struct Layout {
     size_t off_layers, off_pt, off_kc, off_vc, off_h, off_feat, off_abuf, off_qkv, off_attn, off_act, off_po, off_ml,
         off_cnt, off_hp, off_dbgd, off_dbgv, off_out, off_S, off_rlog, off_prompt, off_st, off_bar;
     size_t off_embed, off_head, off_gfinal;
-    size_t off_tmaps;                 // TMA descriptors: 5 per layer / adapter, then the LM head
     std::vector<size_t> off_w[5];     // wqkv, wo, wgate, wup, wdown
     std::vector<size_t> off_g[2];
     size_t total;
@@ -122,7 +120,7 @@ bool valid_config(const kg_config* c) {
     if (c->vocab > (1 << 20) || c->d_ffn > (1 << 20)) return false;      // rows x CTAs must fit 32 bits
     // the plain path stages all rows of an operand in shared memory
     const int kmax = c->d_ffn > c->d_model ? c->d_ffn : c->d_model;
-    const bool plain_somewhere = c->dtype == KG_F32 || c->d_model < 64 || c->d_ffn < 64;
+    const bool plain_somewhere = c->dtype == KG_F32 || (c->d_model % 16) || (c->d_ffn % 16);
     if (plain_somewhere && (size_t)kmax * KG_M_MAX * 4 > (size_t)SIMPLE_XS_BYTES) return false;
     return true;
 }
@@ -169,7 +167,6 @@ Layout make_layout(const kg_config* c, int own_weights, int nctas) {
     L.off_S = take(4 * (size_t)(c->max_seq + KG_M_MAX));
     L.off_rlog = take(16 * (size_t)(c->max_seq + KG_M_MAX));
     L.off_prompt = take(4 * (size_t)c->max_seq);
-    L.off_tmaps = take(sizeof(CUtensorMap) * (size_t)(5 * (nl + 1) + 1));
     for (int k = 0; k < 5; ++k) L.off_w[k].assign(nl + 1, 0);
     for (int k = 0; k < 2; ++k) L.off_g[k].assign(nl + 1, 0);
     L.off_embed = L.off_head = L.off_gfinal = 0;
@@ -201,37 +198,6 @@ int sm_count() {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
     g_sm_count = n;
     return n;
-}
-
-// ---- TMA descriptors of the weight matrices (streamed path) ----------------------------------------------------
-// cuTensorMapEncodeTiled is a driver entry point; it is looked up through the runtime so that the library
-// does not link against the driver.
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-// bf16 matrix [rows][K] row-major -> boxes of 64 k-elements x box_rows rows, 128-byte swizzle, zero fill outside
-int make_weight_map(CUtensorMap* out, const void* W, int rows, int K, int box_rows) {
-    EncodeTiledFn enc = encode_tiled();
-    if (!enc) return KG_E_CUDA;
-    if ((reinterpret_cast<size_t>(W) & 15) || (K % 8) || K < 64 || box_rows < 8 || box_rows > 256) return KG_E_ARG;
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    const cuuint32_t es[2] = {1, 1};
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(W), dims, strides, box, es,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? KG_OK : KG_E_CUDA;
 }
 
 }  // namespace
@@ -379,7 +345,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     D.abuf_pk = (unsigned char*)P(lay.off_abufpk);
     D.ssq_hA = (float*)P(lay.off_ssqA); D.ssq_hB = (float*)P(lay.off_ssqB);
     D.ssq_feat = (float*)P(lay.off_ssqF); D.ssq_abuf = (float*)P(lay.off_ssqAb);
-    D.dm.stream = (cfg->dtype == KG_BF16 && cfg->d_model >= 64 && cfg->d_ffn >= 64) ? 1 : 0;
+    D.dm.stream = (cfg->dtype == KG_BF16 && cfg->d_model % 16 == 0 && cfg->d_ffn % 16 == 0) ? 1 : 0;
     D.dbg_draft = cfg->debug_logits ? (float*)P(lay.off_dbgd) : nullptr;
     D.dbg_verify = cfg->debug_logits ? (float*)P(lay.off_dbgv) : nullptr;
     D.out_tokens = (int*)P(lay.off_out); D.S = (int*)P(lay.off_S); D.round_log = (int*)P(lay.off_rlog);
@@ -410,30 +376,6 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
         }
     }
     cudaStream_t s = m->stream;
-    std::vector<CUtensorMap> tmaps;
-    if (D.dm.stream) {
-        // one descriptor per matrix; the box height is the tile height of the operator's split over the CTAs
-        tmaps.resize(5 * (nl + 1) + 1);
-        CUtensorMap* dev_maps = (CUtensorMap*)P(lay.off_tmaps);
-        const int d = cfg->d_model, F = cfg->d_ffn;
-        int r = KG_OK;
-        for (int i = 0; i <= nl && r == KG_OK; ++i) {
-            LayerW& lw = m->layers_host[i];
-            r = make_weight_map(&tmaps[5 * i + 0], lw.wqkv, 3 * d, d, tc_geom(3 * d, nctas).R);
-            if (r == KG_OK) r = make_weight_map(&tmaps[5 * i + 1], lw.wo, d, d, tc_geom(d, nctas).R);
-            lw.tm_qkv = dev_maps + 5 * i + 0; lw.tm_o = dev_maps + 5 * i + 1;
-            if (i < nl) {
-                if (r == KG_OK) r = make_weight_map(&tmaps[5 * i + 2], lw.wgate, F, d, tc_geom(F, nctas).R);
-                if (r == KG_OK) r = make_weight_map(&tmaps[5 * i + 3], lw.wup, F, d, tc_geom(F, nctas).R);
-                if (r == KG_OK) r = make_weight_map(&tmaps[5 * i + 4], lw.wdown, d, F, tc_geom(d, nctas).R);
-                lw.tm_gate = dev_maps + 5 * i + 2; lw.tm_up = dev_maps + 5 * i + 3; lw.tm_down = dev_maps + 5 * i + 4;
-            }
-        }
-        if (r == KG_OK) r = make_weight_map(&tmaps[5 * (nl + 1)], D.head, cfg->vocab, d, tc_geom(cfg->vocab, nctas).R);
-        D.tm_head = dev_maps + 5 * (nl + 1);
-        if (r != KG_OK) { delete m; return r; }
-        if (cudaMemcpyAsync(dev_maps, tmaps.data(), sizeof(CUtensorMap) * tmaps.size(), cudaMemcpyHostToDevice, s) != cudaSuccess) { delete m; return KG_E_CUDA; }
-    }
     bool ok = cudaMemcpyAsync(P(lay.off_layers), m->layers_host.data(), sizeof(LayerW) * (nl + 1), cudaMemcpyHostToDevice, s) == cudaSuccess;
     // page table: identity, or a fixed permutation (reversal within blocks of 4 pages plus a rotation)
     std::vector<int> pt(D.dm.n_pages);
@@ -814,28 +756,22 @@ OpScratch op_layout() {
     return s;
 }
 
-// the TMA descriptors of the streamed path travel as kernel parameters
 template <typename WT>
-__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int stream, const __grid_constant__ CUtensorMap tm0,
-                                                                     const __grid_constant__ CUtensorMap tm1) {
-    extern __shared__ __align__(1024) char smem[];
-    Ctx& c = ctx_init(smem, nullptr, nullptr, false, stream != 0);
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) op_linear_kernel(LinArgs a, int stream) {
+    extern __shared__ __align__(128) char smem[];
+    Ctx& c = ctx_init(smem, nullptr, nullptr, false);
     OpTable* t = reinterpret_cast<OpTable*>(c.producer ? c.ctl->tab_prod : c.ctl->tab_cons);
-    if (c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0) {
-        t->lin[0] = a;
-        t->lin[0].tmW = &tm0; t->lin[0].tmW2 = a.W2 ? &tm1 : nullptr; t->lin[0].tm_global = 0;
-    }
+    if (c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0) t->lin[0] = a;
     const bool ok = linear_op<WT>(&t->lin[0], c, stream != 0, true);
     if (!ok && c.producer) ring_drain(c);
-    ctx_fini(c, stream != 0);
 }
 __global__ void op_head_final_kernel(const float4* part, int nctas, int M, int* tok, float* p) {
     if (threadIdx.x < M) { int t; float pp; head_final(part, nctas, threadIdx.x, t, pp); tok[threadIdx.x] = t; p[threadIdx.x] = pp; }
 }
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) op_attention_kernel(const __grid_constant__ Dev D, AttArgs a) {
-    extern __shared__ __align__(1024) char smem[];
-    Ctx& c = ctx_init(smem, nullptr, nullptr, false, false);
+    extern __shared__ __align__(128) char smem[];
+    Ctx& c = ctx_init(smem, nullptr, nullptr, false);
     if (!c.producer) {
         OpTable* t = reinterpret_cast<OpTable*>(c.ctl->tab_cons);
         if (threadIdx.x == 0) t->att = a;
@@ -861,27 +797,20 @@ extern "C" int kg_debug_force_simple_ops(int on) { g_force_simple_ops = on ? 1 :
 static int op_linear_common(int32_t dtype, LinArgs& a, unsigned char* xpk, int xpk_k_max, float* ssq, cudaStream_t s) {
     if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
     if (a.M < 1 || a.M > KG_M_MAX || a.N < 1 || a.N > (1 << 20) || a.K < 8 || (a.K % 8)) return KG_E_ARG;
-    const bool plain = dtype == KG_F32 || g_force_simple_ops || a.K < 64 || a.N < 8 || (reinterpret_cast<size_t>(a.W) & 15) ||
-                       (a.W2 && (reinterpret_cast<size_t>(a.W2) & 15));
+    const bool plain = dtype == KG_F32 || g_force_simple_ops || (a.K % 16);
     if (plain && (size_t)a.K * a.M * 4 > (size_t)SIMPLE_XS_BYTES) return KG_E_ARG;
     const int nctas = sm_count();
-    CUtensorMap tm0, tm1;
-    std::memset(&tm0, 0, sizeof(tm0)); std::memset(&tm1, 0, sizeof(tm1));
     if (!plain) {
         if (a.K > xpk_k_max || nctas > 1024) return KG_E_LIMIT;
-        const int box_rows = tc_geom(a.N, nctas).R;
-        int r = make_weight_map(&tm0, a.W, a.N, a.K, box_rows);
-        if (r == KG_OK && a.W2) r = make_weight_map(&tm1, a.W2, a.N, a.K, box_rows);
-        if (r != KG_OK) return r;
         pack_rows_kernel<<<nctas, 256, 0, s>>>(a.x, a.ldx, a.M, a.K, a.gain, xpk, a.K * 4, a.gain ? ssq : nullptr, nctas);
         a.xpk = xpk; a.ldpk = a.K * 4; a.ssq_in = a.gain ? ssq : nullptr;
     }
     if (dtype == KG_BF16) {
         if (set_smem(op_linear_kernel<__nv_bfloat16>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, plain ? 0 : 1, tm0, tm1);
+        op_linear_kernel<__nv_bfloat16><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, plain ? 0 : 1);
     } else {
         if (set_smem(op_linear_kernel<float>) != KG_OK) return KG_E_CUDA;
-        op_linear_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, 0, tm0, tm1);
+        op_linear_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, 0);
     }
     CK(cudaGetLastError());
     return KG_OK;

@@ -7,14 +7,12 @@
 //
 // A CTA has 8 consumer warps and one producer warp.  The decode step is bound by HBM bandwidth:
 // every weight byte is read exactly once per pass.  The producer warp streams this CTA's share of
-// every weight matrix of a pass through a ring of shared-memory slots with TMA tile copies
-// (cp.async.bulk.tensor, 128-byte swizzle, mbarrier transaction counts); because weights do not
-// depend on activations it runs ahead of the consumers across operator boundaries and grid
-// barriers, so HBM stays busy while the consumers synchronise.  One consumer thread feeds the
-// 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory) straight from the ring:
-// the "M" side of an MMA is a tile of up to 96 weight rows, the "N" side the 1..16 activation rows,
-// split into bf16 hi + lo so that the product keeps fp32 accuracy.  The other consumer warps stage
-// the activation operand in shared memory ahead of the MMAs and run the epilogues.
+// every weight matrix of a pass through a ring of shared-memory slots with bulk asynchronous
+// copies (cp.async.bulk + mbarrier transaction counts); because weights do not depend on
+// activations it runs ahead of the consumers across operator boundaries and grid barriers, so HBM
+// stays busy while the consumers synchronise.  The consumers read weight tiles with ldmatrix and
+// feed tensor-core MMAs whose "M" side is the weight tile and whose "N" side is the 1..16
+// activation rows (activations split into bf16 hi + lo so that the product keeps fp32 accuracy).
 #pragma once
 
 #include <cuda_bf16.h>
@@ -38,34 +36,20 @@ constexpr int BLOCK_THREADS = NTHREADS + 32;   // + the producer warp (warp inde
 constexpr int S_CAP = 16;          // most KV splits per head
 constexpr int HD_MAX = 128;
 
-// weight ring: RING slots; a stage is A "atoms" of one weight tile, an atom being R rows x 64 k-elements (128 bytes
-// per row, 128-byte swizzle: the canonical K-major operand layout of tcgen05.mma), R * A * 128 <= SLOT_BYTES
-constexpr int RING = 7;
-constexpr int SLOT_BYTES = 24576;
-constexpr int TILE_ROWS_MAX = 96;                       // weight rows per MMA tile (M = 128 MMAs; the rows above R are ignored)
+// weight ring: RING slots of ST_ROWS weight rows x ST_K k-elements (bf16); rows are padded by 16
+// bytes so that the eight row addresses of an ldmatrix fall into distinct bank groups
+constexpr int RING = 6;
+constexpr int ST_ROWS = 8;
+constexpr int ST_K = 2048;
+constexpr int ST_ROW_BYTES = ST_K * 2 + 16;
+constexpr int SLOT_BYTES = ST_ROWS * ST_ROW_BYTES;
 constexpr int CTRL_BYTES = 3072;
 constexpr int OP_TABLE_BYTES = 1024;                    // struct OpTable: the operator arguments of one layer
 constexpr int RING_OFF = CTRL_BYTES;
-// activation operand (B): NB buffers of BBUF_BYTES, one per k phase, filled ahead of the MMAs
-constexpr int NB = 6;
-constexpr int BBUF_BYTES = 8192;
-constexpr int BBUF_OFF = RING_OFF + RING * SLOT_BYTES;
-constexpr int WORK_OFF = BBUF_OFF + NB * BBUF_BYTES;
+constexpr int WORK_OFF = RING_OFF + RING * SLOT_BYTES;
 constexpr int SMEM_TOTAL = 232448;                      // 227 KB, the most one CTA may own
-constexpr int WORK_BYTES = SMEM_TOTAL - WORK_OFF;       // small per-operator tables (1/rms, prefetched residuals, ...)
-// The accumulators of a superchunk leave tensor memory through the B buffers (idle by then); attention, which never
-// overlaps a linear operator inside a CTA, uses the same bytes.
-constexpr int MP = 16;                                  // accumulator columns (activation rows, padded)
-constexpr int ACC_ROWS = NB * BBUF_BYTES / (MP * 4);    // 768 accumulator rows
-constexpr int TMEM_COLS = 512;                          // tensor-memory columns held by the CTA (all of them)
-// The tensor core adds into an fp32 accumulator with truncation, so a long chain of MMAs on one accumulator drifts
-// (measured: a shrink of about 2e-8 of the sum per MMA).  Successive k16-steps therefore rotate over all accumulators the
-// tensor memory has room for (32 per weight tile for M <= 8 rows, half of that for the SwiGLU pair or M > 8), which the
-// epilogue adds in fp32 with rounding.  One unit tile accumulates at a time.
-constexpr int ACC2_ROWS = 384;                          // the two halves of the accumulator sums sit this many rows apart
-constexpr int B_AHEAD = 3;                              // phases whose activation loads may be in flight
-static_assert(RING_OFF % 1024 == 0 && SLOT_BYTES % 1024 == 0 && BBUF_BYTES % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
-static_assert(B_AHEAD < NB - 1, "activation buffers");
+constexpr int WORK_BYTES = SMEM_TOTAL - WORK_OFF;       // activations, reductions, attention tiles
+constexpr int SC_ROWS = 256;                            // rows whose accumulators live in shared memory at once
 // the plain path never runs beside the streamed one in a launch, so it stages its activations over the ring too
 constexpr int SIMPLE_XS_BYTES = SMEM_TOTAL - RING_OFF - 4096;
 
@@ -79,8 +63,6 @@ enum { ST_OK = 0, ST_TIMEOUT = -6 };
 struct LayerW {
     const void* wqkv; const void* wo; const void* wgate; const void* wup; const void* wdown;
     const float* g1; const float* g2;
-    // TMA descriptors of the five matrices (streamed path), in global memory
-    const void* tm_qkv; const void* tm_o; const void* tm_gate; const void* tm_up; const void* tm_down;
 };
 
 struct Dims {
@@ -88,7 +70,7 @@ struct Dims {
     float eps, theta, logit_scale;
     int max_seq, page_size, n_pages, gamma_max, debug;
     int ps_shift;       // log2(page_size): page sizes are powers of two
-    int stream;         // 1: linear operators take the streamed tensor-core path (bf16 weights)
+    int stream;         // 1: linear operators take the streamed tensor-core path (bf16, d and F multiples of 16)
 };
 
 // Device-resident sequence / round state (one int-sized field per line of the method's notation).
@@ -114,7 +96,6 @@ struct State {
 struct Dev {
     Dims dm;
     const void* embed; const void* head; const float* g_final;
-    const void* tm_head;           // TMA descriptor of the LM head (streamed path)
     const LayerW* layers;          // [L+1], index L = adapter
     void* kcache; void* vcache;    // [(L+1)][n_pages][H][page_size][hd]
     const int* page_table;         // [n_pages] logical -> physical page
@@ -124,7 +105,7 @@ struct Dev {
     float* qkv;                    // [M_MAX][3d]
     float* attn;                   // [M_MAX][d]
     float* act;                    // [M_MAX][F]
-    // packed copies (streamed path; row = K bf16 hi values, then K bf16 lo values) and per-CTA sums of squares [row][nctas]
+    // packed copies (streamed path; row = 4 bytes per element) and per-CTA sums of squares [row][nctas]
     unsigned char* hA_pk;          // [M_MAX][d]   residual stream scaled for the next QKV / the LM head
     unsigned char* hB_pk;          // [M_MAX][d]   residual stream after attention scaled for the SwiGLU pair
     unsigned char* attn_pk;        // [M_MAX][d]
@@ -149,12 +130,8 @@ struct Dev {
 
 // Per-CTA control block at the start of shared memory.
 struct Ctrl {
-    unsigned long long full[RING];     // producer -> MMA issuer: slot filled (transaction count)
-    unsigned long long empty[RING];    // tensor core -> producer: the MMAs that read the slot have completed
-    unsigned long long bready[NB];     // loaders -> MMA issuer: activation buffer filled
-    unsigned long long bfree[NB];      // tensor core -> loaders: the MMAs that read the buffer have completed
-    unsigned long long done;           // tensor core -> consumers: the accumulators of a superchunk are final
-    unsigned tmem_base;                // tensor-memory address of the CTA's accumulator columns
+    unsigned long long full[RING];     // producer -> consumers: slot filled (transaction count)
+    unsigned long long empty[RING];    // consumers -> producer: slot drained (one arrival per consumer warp)
     unsigned long long mail;           // consumers -> producer: head_tok / head_p hold a new result
     int abort;                         // a bounded wait of this CTA gave up
     int sync_ok;
@@ -184,8 +161,6 @@ struct Ctx {
     bool grid;                     // false: single-operator test kernel, grid barriers are CTA barriers
     bool producer;                 // this thread belongs to the producer warp
     int slot; unsigned phase;      // ring cursor of this thread's role
-    unsigned bph;                  // consumers: activation phases so far (buffer = bph % NB, its use index = bph / NB)
-    unsigned done_cnt;             // consumers: completed superchunks so far
     unsigned issued;               // producer: stages issued so far
     unsigned mail_phase;           // producer: parity of the next result it waits for
 };
@@ -221,56 +196,11 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// ---- TMA tile copy, tensor memory and tcgen05 MMA ----------------------------------------------------------------
-// One box of a 2-D tensor map (64 k-elements x R rows, 128-byte swizzle) -> shared memory; x is a multiple of 64 elements.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap, int x, int y, uint32_t bar_smem) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst_smem), "l"(tmap), "r"(x), "r"(y), "r"(bar_smem) : "memory");
+// global -> shared bulk copy; bytes and both addresses are multiples of 16
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsigned bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// a tensor map that lives in global memory is acquired once before the copies that use it
-__device__ __forceinline__ void tmap_acquire(const void* tmap) {
-    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory operand descriptor: K-major, 128-byte swizzle (rows of 128 bytes, groups of 8 rows 1024 bytes apart).
-// bits [0,14) address >> 4, [16,30) leading offset >> 4 (unused here), [32,46) group stride >> 4, [46,48) version 1,
-// [61,64) layout 2 = 128-byte swizzle.  Stepping 16 k-elements inside the 64-element atom adds 32 bytes to the address.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
-    const uint32_t lo = ((saddr & 0x3FFFFu) >> 4) | (1u << 16);
-    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    return ((uint64_t)hi << 32) | lo;
-}
-// Instruction descriptor: fp32 accumulate (bit 4), bf16 A and B (bits 7, 10), both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
-__device__ __forceinline__ uint32_t umma_idesc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
-}
-// D[128 x N] (+)= A[128 x 16] B[N x 16]^T, issued by one thread
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// the mbarrier receives one arrival when every MMA this thread has issued so far has completed
-__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// 64 consecutive accumulator columns of this thread's tensor-memory lane (lane = 32 * (warp % 4) + lane id)
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
-    uint32_t r[64];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n\t"
-                 "tcgen05.wait::ld.sync.aligned;"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
-                 : "r"(taddr) : "memory");
-#pragma unroll
-    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void record_timeout(Ctx& c, int where) {
     *(volatile int*)&c.ctl->abort = 1;
@@ -294,6 +224,16 @@ __device__ __forceinline__ bool mbar_wait(Ctx& c, unsigned long long* bar, unsig
         }
     }
     return true;
+}
+
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -328,9 +268,8 @@ __device__ __forceinline__ bool arg_better(float za, int ia, float zb, int ib) {
 }
 
 // ------------------------------------------------------------------------------------ CTA set-up
-// Called by every thread of the CTA at kernel start; returns the context of the thread's role.  tc: the launch
-// uses the streamed tensor-core path, so the CTA takes its tensor-memory columns (ctx_fini gives them back).
-__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, bool grid, bool tc) {
+// Called by every thread of the CTA at kernel start; returns the context of the thread's role.
+__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, bool grid) {
     static_assert(sizeof(Ctx) <= 128, "context slot too small");
     Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
     const bool producer = threadIdx.x >= NTHREADS;
@@ -339,44 +278,17 @@ __device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, b
         c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
         c.ctl = ctl; c.grid = grid;
         c.producer = producer;
-        c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0; c.bph = 0; c.done_cnt = 0;
+        c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0;
     }
     KG_PROBE_INIT();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < RING; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        for (int i = 0; i < NB; ++i) { mbar_init(&ctl->bready[i], NTHREADS - 32); mbar_init(&ctl->bfree[i], 1); }
-        mbar_init(&ctl->done, 1);
+        for (int i = 0; i < RING; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], NWARPS); }
         mbar_init(&ctl->mail, 1);
-        ctl->abort = 0; ctl->sync_ok = 1; ctl->att_last = 0; ctl->tmem_base = 0;
-        // swizzled tiles need the ring on a 1024-byte boundary of the shared window
-        if (tc && (smem_u32(smem) & 1023u) != 0u) {
-            ctl->abort = 1;
-            if (st) atomicCAS(&st->status, 0, ST_TIMEOUT);
-        }
+        ctl->abort = 0; ctl->sync_ok = 1; ctl->att_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (tc) {
-        if (threadIdx.x < 32) {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(TMEM_COLS) : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-    }
     return c;
-}
-
-// Called by every thread of the CTA before the kernel returns.
-__device__ __forceinline__ void ctx_fini(Ctx& c, bool tc) {
-    if (!tc) return;
-    tc_fence_before();
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.ctl->tmem_base), "r"(TMEM_COLS) : "memory");
-    }
 }
 
 // ------------------------------------------------------------------------------------ grid barrier
@@ -424,28 +336,32 @@ __device__ __forceinline__ void rope_cs(const Dev& D, int pos, int i, float& cs,
 }
 
 // ------------------------------------------------------------------------------------ linear operator
-// A packed copy of an activation row of K elements: K bf16 "hi" values followed by K bf16 "lo" values with
-// x * gain = hi + lo (gain: the norm gain of the operator that reads the row).  The operator that produces a
-// row writes it once in this form; the reader copies 16-byte pieces of it into the swizzled operand tile.
+// A packed copy of activation rows: the row is cut into k16 blocks of 64 bytes; the 16 bytes at
+// blk*64 + tt*16 hold {hi(k), hi(k+8), lo(k), lo(k+8)} for k = 16 blk + 2 tt, each a pair of bf16
+// (elements k, k+1) with x * gain = hi + lo.  This is the B operand fragment order of the MMA, so a
+// consumer lane fetches its fragments with plain 8- or 16-byte loads.  The operator that produces a
+// row writes it once, in this form, for the operator that reads it.
 struct PkOut { const float* gain; unsigned char* ptr; };   // gain == null: unscaled
 
-__device__ __forceinline__ void pk_store(unsigned char* row, int K, int k, float v) {
+// byte offset of the hi half of element k inside a packed row; the lo half sits 8 bytes further
+__device__ __forceinline__ size_t pk_off(int k) {
+    return (size_t)(k >> 4) * 64 + (size_t)(((k & 7) >> 1) * 16 + ((k >> 3) & 1) * 4 + (k & 1) * 2);
+}
+__device__ __forceinline__ void pk_store(unsigned char* row, int k, float v) {
     const __nv_bfloat16 h = __float2bfloat16_rn(v);
     const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
-    __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(row);
-    p[k] = h;
-    p[K + k] = l;
+    unsigned char* p = row + pk_off(k);
+    *reinterpret_cast<__nv_bfloat16*>(p) = h;
+    *reinterpret_cast<__nv_bfloat16*>(p + 8) = l;
 }
 
 struct LinArgs {
     const void* W; const void* W2;   // [N, K]; W2 != null: SwiGLU pair (gate, up)
-    const void* tmW; const void* tmW2;   // streamed path: TMA descriptors of W, W2 (box = 64 k-elements x tc_geom().R rows)
-    int tm_global;                   // the descriptors live in global memory (acquired before use)
     int N, K;
     int M;                           // activation rows
     const float* x; int ldx;         // plain path: fp32 rows (written earlier in this kernel)
     const float* gain; float eps;    // RMSNorm gain of the input (null: no norm)
-    const unsigned char* xpk; int ldpk;   // streamed path: packed rows, already multiplied by the gain; bytes per row (4 K)
+    const unsigned char* xpk; int ldpk;   // streamed path: packed rows, already multiplied by the gain; bytes per row
     const float* ssq_in;             // streamed path with norm: [M][nctas] partial sums of squares of the input rows
     const float* resid; int ldr;     // EPI_RESID
     float* out; int ldo;             // fp32 output rows (streamed path: nullable)
@@ -472,95 +388,81 @@ __device__ __forceinline__ void head_merge(HeadStat& a, float zmax, float sum, i
     }
 }
 
-// ---- streamed tensor-core path (bf16 weights, K a multiple of 8) ------------------------------------
+// ---- streamed tensor-core path (bf16 weights, K a multiple of 16) -----------------------------------
 //
 // Work split.  The CTA owns a contiguous range of "units": output rows, or for the SwiGLU pair
-// gate/up feature pairs.  The range is cut into tiles of at most 96 units; a tile's weights are the
-// A operand of M = 128 MMAs (tensor-memory lanes above the tile's rows hold garbage that is never
-// read).  The activations are the B operand with N = 16 (M <= 8 rows: hi in B rows 0-7, lo in 8-15)
-// or N = 32 columns; D[:, m] + D[:, N/2 + m] is the product with activation row m.
+// gate/up feature pairs.  A stage of the ring holds 8 weight rows (for the pair: the 8 gate rows of
+// a feature group, then in the next stage the 8 up rows of the same features) times one k phase
+// (2048 k-elements when M <= 8, else 1024), i.e. one bulk copy of up to 4 KB per row: the copy
+// engine spends a fixed time per copy, and only copies of 2-4 KB and more keep HBM saturated.
+// The stages are visited superchunk (<= 256 accumulator rows) -> phase -> row group, in the same
+// order by the producer warp (which issues the copies) and the consumers.
 //
-// k is walked in phases of PA atoms (an atom = 64 k-elements); the B operand of a phase sits in one
-// of NB shared-memory buffers that the loader warps fill a few phases ahead.  Inside a phase the
-// stages are visited tile -> (gate, up) -> chunk of A atoms, in the same order by the producer warp
-// (which issues one TMA box per atom) and by the MMA issuer.  All tiles of a superchunk (up to four
-// weight tiles) accumulate in tensor memory at once; after the last phase the accumulators are
-// copied to shared memory and the epilogue runs as one pass over the superchunk.
-struct TcGeom { int per, nt, rt, R, A; };
-// units per CTA (most), tiles, units per tile, rows of a TMA box (rt rounded up to 8), atoms per stage
-__host__ __device__ inline TcGeom tc_geom(int n_units, int nctas) {
-    TcGeom g;
-    g.per = (n_units + nctas - 1) / nctas;
-    g.nt = (g.per + TILE_ROWS_MAX - 1) / TILE_ROWS_MAX;
-    if (g.nt < 1) g.nt = 1;
-    g.rt = (g.per + g.nt - 1) / g.nt;
-    if (g.rt < 1) g.rt = 1;
-    g.R = (g.rt + 7) & ~7;
-    g.A = g.R <= 24 ? 8 : (g.R <= 48 ? 4 : 2);
-    return g;
-}
+// Consumers take the stages two at a time: one MMA m16n8k16 computes D[weight row, activation
+// column] with the 16 weight rows of a stage pair as the A operand (ldmatrix straight from the
+// ring) and the activations as the 8-column B operand.  The activations keep fp32 accuracy by a
+// split x * gain = hi + lo into two bf16 parts:
+//   V = 4  (M <= 4):  columns 0-3 carry hi, columns 4-7 lo of rows 0-3: one MMA per k16-step;
+//   V = 8  (M <= 8):  hi and lo are two MMAs;
+//   V = 16 (M <= 16): two column tiles, hi and lo: four MMAs.
+// Each of the 8 warps owns a fixed slice of the phase's k range; its B fragments are loaded once
+// per phase from the packed activation rows in global memory (L2) and stay in registers for every
+// row group, so the steady state touches shared memory only for the weights.  After a stage pair the 8 partial sums of each (weight row,
+// activation row) are added in warp order into the per-row accumulators in shared memory.
+template <int V> struct LinGeom {
+    static constexpr int NS = V == 16 ? 8 : 16;           // k16-steps per warp and stage
+    static constexpr int PLEN = NS * 16 * NWARPS;         // k-elements per phase: 2048 or 1024
+    static constexpr int FR = V == 4 ? 2 : (V == 8 ? 4 : 8);   // B fragment registers per step
+    static constexpr int NACC = V == 16 ? 2 : 1;          // column tiles
+};
+constexpr int MP = 16;                                    // accumulator columns (activation rows, padded)
 
-struct TcPlan {
+struct LinPlan {
     int u0, u1;          // this CTA's units
-    int nt, rt, R, A;    // unit tiles, units per tile, box rows, atoms per stage
-    int N, PA;           // B rows; atoms per phase
-    int G;               // accumulators per weight tile (a power of two)
-    int natoms, nph;     // atoms of K; phases
-    int tps;             // unit tiles per superchunk
-    int wtiles;          // weight tiles per unit tile (2 for the SwiGLU pair)
+    int sc_units;        // units per superchunk
+    int plen, nph;       // k phases
 };
 
-__device__ __forceinline__ TcPlan tc_plan(const LinArgs& a, int cta, int nctas) {
-    TcPlan p;
+__device__ __forceinline__ LinPlan make_plan(const LinArgs& a, int cta, int nctas) {
+    LinPlan p;
     p.u0 = (int)((unsigned)a.N * (unsigned)cta / (unsigned)nctas);          // N * nctas < 2^32 (checked on the host)
     p.u1 = (int)((unsigned)a.N * (unsigned)(cta + 1) / (unsigned)nctas);
-    const TcGeom g = tc_geom(a.N, nctas);
-    p.nt = g.nt; p.rt = g.rt; p.R = g.R;
-    p.N = a.M <= 8 ? 16 : 32;
-    p.PA = BBUF_BYTES / (p.N * 128);
-    p.A = min(g.A, p.PA);
-    p.natoms = (a.K + 63) >> 6;
-    p.nph = (p.natoms + p.PA - 1) / p.PA;
-    p.wtiles = a.W2 ? 2 : 1;
-    p.tps = 1;
-    p.G = TMEM_COLS / (p.N * p.wtiles);
+    p.sc_units = a.W2 ? SC_ROWS / 2 : SC_ROWS;
+    p.plen = a.M <= 8 ? LinGeom<8>::PLEN : LinGeom<16>::PLEN;
+    p.nph = (a.K + p.plen - 1) / p.plen;
     return p;
 }
 
-// Producer warp: issue the TMA copies of every stage of this operator.
+// Producer warp: issue the bulk copies of every stage of this operator.
 __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
     const int lane = threadIdx.x & 31;
-    const TcPlan pl = tc_plan(a, c.cta, c.nctas);
+    const LinPlan pl = make_plan(a, c.cta, c.nctas);
+    const bool dual = a.W2 != nullptr;
+    const __nv_bfloat16* W = reinterpret_cast<const __nv_bfloat16*>(a.W);
+    const __nv_bfloat16* W2 = reinterpret_cast<const __nv_bfloat16*>(a.W2);
+    char* ring = c.smem + RING_OFF;
     Ctrl* ctl = c.ctl;
-    const uint32_t ring = smem_u32(c.smem + RING_OFF);
     int slot = c.slot; unsigned phase = c.phase; unsigned issued = c.issued;     // ring cursor, kept in registers here
-    if (a.tm_global && lane == 0) { tmap_acquire(a.tmW); if (a.tmW2) tmap_acquire(a.tmW2); }
-    __syncwarp();
-    for (int t0 = 0; t0 < pl.nt; t0 += pl.tps) {
-        const int t1 = min(pl.nt, t0 + pl.tps);
+    for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
+        const int sc1 = min(pl.u1, sc0 + pl.sc_units);
+        const int ngrp = (sc1 - sc0 + ST_ROWS - 1) / ST_ROWS;
+        const int nst = dual ? 2 * ngrp : ngrp;
         for (int ph = 0; ph < pl.nph; ++ph) {
-            const int a0 = ph * pl.PA, a1 = min(pl.natoms, a0 + pl.PA);
-            for (int t = t0; t < t1; ++t) {
-                const int row0 = pl.u0 + t * pl.rt;
-                if (row0 >= pl.u1) continue;
-                for (int w = 0; w < pl.wtiles; ++w) {
-                    const void* tm = w ? a.tmW2 : a.tmW;
-                    for (int at = a0; at < a1; at += pl.A) {
-                        const int n_at = min(pl.A, a1 - at);
-                        int ok = 1;
-                        if (lane == 0) ok = mbar_wait(c, &ctl->empty[slot], phase ^ 1u, 40) ? 1 : 0;
-                        ok = __shfl_sync(0xffffffffu, ok, 0);
-                        if (!ok) { c.slot = slot; c.phase = phase; c.issued = issued; return false; }
-                        if (lane == 0) mbar_arrive_expect_tx(&ctl->full[slot], (unsigned)(n_at * pl.R * 128));
-                        __syncwarp();
-                        if (lane < n_at)
-                            tma_load_2d(ring + (uint32_t)slot * SLOT_BYTES + (uint32_t)(lane * pl.R * 128), tm, (at + lane) * 64, row0,
-                                        smem_u32(&ctl->full[slot]));
-                        KG_PROBE(30);
-                        issued++;
-                        if (++slot == RING) { slot = 0; phase ^= 1u; }
-                    }
-                }
+            const int p0 = ph * pl.plen, len = min(pl.plen, a.K - p0);
+            for (int si = 0; si < nst; ++si) {
+                const int base = sc0 + (dual ? si >> 1 : si) * ST_ROWS;
+                const int nvalid = min(ST_ROWS, sc1 - base);
+                const __nv_bfloat16* src = ((dual && (si & 1)) ? W2 : W) + (size_t)(base + lane) * a.K + p0;
+                int ok = 1;
+                if (lane == 0) ok = mbar_wait(c, &ctl->empty[slot], phase ^ 1u, 40) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { c.slot = slot; c.phase = phase; c.issued = issued; return false; }
+                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[slot], (unsigned)(nvalid * len * 2));
+                __syncwarp();
+                if (lane < nvalid) bulk_g2s(ring + (size_t)slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &ctl->full[slot]);
+                KG_PROBE(30);
+                issued++;
+                if (++slot == RING) { slot = 0; phase ^= 1u; }
             }
         }
     }
@@ -582,8 +484,18 @@ __device__ void ring_drain(Ctx& c) {
     }
 }
 
-// Shared-memory tables of the streamed path (floats, from WORK_OFF).
-constexpr int LW_RS = 0;                                  // [M_MAX] 1/rms of the input rows
+__device__ __forceinline__ void split_hi_lo(float2 v, unsigned& hi, unsigned& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(v.x, v.y);
+    const float2 f = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(v.x - f.x, v.y - f.y);
+    hi = *reinterpret_cast<const unsigned*>(&h);
+    lo = *reinterpret_cast<const unsigned*>(&l);
+}
+
+// Shared-memory work area of the streamed path (floats, from WORK_OFF).
+constexpr int LW_RED = 0;                                 // [2][NWARPS][16][8] partial sums of a stage pair
+constexpr int LW_ACC = LW_RED + 2 * NWARPS * 128;         // [SC_ROWS][MP] row accumulators
+constexpr int LW_RS = LW_ACC + SC_ROWS * MP;              // [M_MAX] 1/rms of the input rows
 constexpr int LW_RSP = LW_RS + M_MAX;                     // [M_MAX][16] partial sums of squares of the input rows
 constexpr int LW_SSW = LW_RSP + M_MAX * 16;               // [NWARPS][M_MAX] sums of squares of the output rows
 constexpr int PRE_NU = 64;                                // residual / gain values are prefetched for up to this many units
@@ -591,7 +503,6 @@ constexpr int LW_PRES = LW_SSW + NWARPS * M_MAX;          // [M_MAX][PRE_NU] res
 constexpr int LW_PREG = LW_PRES + M_MAX * PRE_NU;         // [2][PRE_NU] gains of the packed outputs
 constexpr int LW_END = LW_PREG + 2 * PRE_NU;
 static_assert(LW_END * 4 <= WORK_BYTES, "linear work area too large");
-static_assert(2 * TILE_ROWS_MAX <= ACC2_ROWS && 2 * ACC2_ROWS <= ACC_ROWS, "accumulator rows of a superchunk");
 
 __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
@@ -602,27 +513,24 @@ __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
 // Thread (r, m): m = tid mod 2^ceil(log2 M), so that the lanes of a warp that share m can add their
 // squares by shuffles in a fixed order.  Every consumer thread calls it; ssq_acc (threads < M)
 // accumulates over superchunks.
-__device__ __forceinline__ void emit_rows(const LinArgs& a, const float* acc_s, int acc2, float* wk, int sc0, int nu, bool prefetched, float& ssq_acc) {
-    // acc2: float offset of the second half of the accumulator sums
+__device__ __forceinline__ void emit_rows(const LinArgs& a, float* wk, int sc0, int nu, bool prefetched, float& ssq_acc) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M;
+    const float* acc_s = wk + LW_ACC;
     const float* rs = wk + LW_RS;
     float* ssw = wk + LW_SSW;
     const int sh = M <= 1 ? 0 : (M <= 2 ? 1 : (M <= 4 ? 2 : (M <= 8 ? 3 : 4)));
     const int mp = 1 << sh;
     const int m = tid & (mp - 1);
-    const int Kout = a.ldpk_out >> 2;                        // elements of a packed output row
     float ssl = 0.f;
     if (m < M) {
         for (int r = tid >> sh; r < nu; r += NTHREADS >> sh) {
             float v;
             if (a.epi == EPI_SWIGLU) {
                 const int srow = (r >> 3) * 16 + (r & 7);
-                const float gt = acc_s[(size_t)srow * MP + m] + acc_s[acc2 + (size_t)srow * MP + m];
-                const float up = acc_s[(size_t)(srow + 8) * MP + m] + acc_s[acc2 + (size_t)(srow + 8) * MP + m];
-                v = silu_f(gt * rs[m]) * (up * rs[m]);
+                v = silu_f(acc_s[(size_t)srow * MP + m] * rs[m]) * (acc_s[(size_t)(srow + 8) * MP + m] * rs[m]);
             } else {
-                v = (acc_s[(size_t)r * MP + m] + acc_s[acc2 + (size_t)r * MP + m]) * rs[m];
+                v = acc_s[(size_t)r * MP + m] * rs[m];
                 if (a.epi == EPI_RESID)
                     v += prefetched ? wk[LW_PRES + m * PRE_NU + r] : ldcg_f(a.resid + (size_t)m * a.ldr + sc0 + r);
             }
@@ -634,7 +542,7 @@ __device__ __forceinline__ void emit_rows(const LinArgs& a, const float* acc_s, 
                 if (a.pk[q].ptr) {
                     float pv = v;
                     if (a.pk[q].gain) pv *= prefetched ? wk[LW_PREG + q * PRE_NU + r] : __ldg(a.pk[q].gain + row);
-                    pk_store(a.pk[q].ptr + (size_t)m * a.ldpk_out, Kout, row, pv);
+                    pk_store(a.pk[q].ptr + (size_t)m * a.ldpk_out, row, pv);
                 }
             }
         }
@@ -651,202 +559,202 @@ __device__ __forceinline__ void emit_rows(const LinArgs& a, const float* acc_s, 
     }
 }
 
-// Consumer warps of one streamed operator.  Warp 0: its first lane issues the MMAs; warps 1-7: fill the
-// activation buffers ahead of them; all eight: epilogue.
+template <int V>
 __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
-    constexpr int NLOAD = NTHREADS - 32;                                    // loader threads
+    using G = LinGeom<V>;
+    constexpr int NS = G::NS, FR = G::FR, NACC = G::NACC;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
     const int M = a.M, K = a.K;
-    const TcPlan pl = tc_plan(a, c.cta, c.nctas);
     const bool dual = a.W2 != nullptr;
+    const LinPlan pl = make_plan(a, c.cta, c.nctas);
 
     float* wk = reinterpret_cast<float*>(c.smem + WORK_OFF);
-    float* acc_s = reinterpret_cast<float*>(c.smem + BBUF_OFF);
+    float* red = wk + LW_RED;
+    float* acc_s = wk + LW_ACC;
     float* rs = wk + LW_RS;
+    const char* ring = c.smem + RING_OFF;
     Ctrl* ctl = c.ctl;
     const int nctas = c.nctas, cta = c.cta;
-    const uint32_t ring = smem_u32(c.smem + RING_OFF);
-    const uint32_t bbuf = smem_u32(c.smem + BBUF_OFF);
-    const uint32_t tmem = ctl->tmem_base;
-    unsigned bph = c.bph, done_cnt = c.done_cnt;                            // the same values in every consumer thread
+    int slot = c.slot; unsigned phase = c.phase;              // ring cursor, kept in registers here
 
     HeadStat hs[2];                                                        // EPI_HEAD: this warp tracks rows warp, warp + 8
     hs[0].zmax = hs[1].zmax = 0.f; hs[0].sum = hs[1].sum = 0.f; hs[0].arg = hs[1].arg = 0;
     bool ok = true;
+    int buf = 0;
     float ssq_acc = 0.f;
     KG_PROBE(10);
 
-    const int nu0 = max(0, min(pl.u1 - pl.u0, pl.tps * pl.rt));             // units of the first superchunk
+    // ---- fetched early, used in the epilogue: the input rows' sums of squares, residual values, output gains.
+    // The requests go out right behind the first phase's fragment loads, which the first MMA waits for.
+    const int nu0 = min(pl.u1 - pl.u0, pl.sc_units);
     const bool prefetched = nu0 <= PRE_NU;
-    bool first = true;
+    bool pre_pending = true;
+    auto epilogue_prefetch = [&]() {
+        if (a.ssq_in) {
+            // thread (m, j) adds the partial sums of CTAs j, j + 16, ... of row m
+            const int m = tid >> 4, j = tid & 15;
+            float part = 0.f;
+            if (m < M) for (int q = j; q < nctas; q += 16) part += ldcg_f(a.ssq_in + (size_t)m * nctas + q);
+            wk[LW_RSP + tid] = part;
+        }
+        if (prefetched && a.epi != EPI_HEAD) {
+            if (a.epi == EPI_RESID)
+                for (int i = tid; i < M * nu0; i += NTHREADS) cp_async4(wk + LW_PRES + (i / nu0) * PRE_NU + i % nu0, a.resid + (size_t)(i / nu0) * a.ldr + pl.u0 + i % nu0);
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+                if (a.pk[q].ptr && a.pk[q].gain)
+                    for (int i = tid; i < nu0; i += NTHREADS) cp_async4(wk + LW_PREG + q * PRE_NU + i, a.pk[q].gain + pl.u0 + i);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
 
-    for (int t0 = 0; t0 < pl.nt; t0 += pl.tps) {
-        const int sc0 = pl.u0 + t0 * pl.rt;
-        if (sc0 >= pl.u1) break;
-        const int t1 = min(pl.nt, t0 + pl.tps);
-        const int sc1 = min(pl.u1, pl.u0 + t1 * pl.rt);
+    // this lane's rows of the packed input: V = 4: row g & 3 (hi for g < 4, lo for g >= 4); else rows g (and g + 8)
+    const int xrow = V == 4 ? (g & 3) : g;
+    const unsigned char* xlane = a.xpk + (size_t)xrow * a.ldpk + (size_t)warp * NS * 64 + t * 16 + (V == 4 ? (g >> 2) * 8 : 0);
+
+    for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
+        const int sc1 = min(pl.u1, sc0 + pl.sc_units);
         const int nu = sc1 - sc0;
-
-        if (warp == 0) {
-            // ---- MMA issuer
-            if (lane == 0) {
-                int slot = c.slot; unsigned phase = c.phase;
-                const uint32_t idesc = umma_idesc(pl.N);
-                for (int ph = 0; ph < pl.nph; ++ph) {
-                    const int a0 = ph * pl.PA, a1 = min(pl.natoms, a0 + pl.PA);
-                    const unsigned gph = bph + (unsigned)ph;
-                    const int buf = (int)(gph % NB);
-                    if (ok) ok = mbar_wait(c, &ctl->bready[buf], (gph / NB) & 1u, 44);
-                    tc_fence_after();
-                    const uint32_t bbase = bbuf + (uint32_t)buf * BBUF_BYTES;
-                    for (int t = t0; t < t1; ++t) {
-                        if (pl.u0 + t * pl.rt >= pl.u1) continue;
-                        for (int w = 0; w < pl.wtiles; ++w) {
-                            const uint32_t dcol = tmem + (uint32_t)(((t - t0) * pl.wtiles + w) * pl.G * pl.N);
-                            for (int at = a0; at < a1; at += pl.A) {
-                                const int n_at = min(pl.A, a1 - at);
-                                if (ok) ok = mbar_wait(c, &ctl->full[slot], phase, 41);
-                                KG_PROBE(12);
-                                if (ok) {
-                                    tc_fence_after();
-                                    const uint32_t abase = ring + (uint32_t)slot * SLOT_BYTES;
-                                    for (int q = 0; q < n_at; ++q) {
-                                        const int k0 = (at + q) * 64;
-                                        const int steps = min(4, (K - k0 + 15) >> 4);
-                                        const uint32_t aaddr = abase + (uint32_t)(q * pl.R * 128);
-                                        const uint32_t baddr = bbase + (uint32_t)((at + q - a0) * pl.N * 128);
-                                        for (int j = 0; j < steps; ++j) {
-                                            const int st = (at + q) * 4 + j;                 // k16-step of the whole row
-                                            umma_bf16(dcol + (uint32_t)((st & (pl.G - 1)) * pl.N), umma_desc(aaddr + j * 32),
-                                                      umma_desc(baddr + j * 32), idesc, st >= pl.G ? 1u : 0u);
-                                        }
-                                    }
-                                    umma_commit(&ctl->empty[slot]);
-                                }
-                                KG_PROBE(13);
-                                if (++slot == RING) { slot = 0; phase ^= 1u; }
+        const int ngrp = (nu + ST_ROWS - 1) / ST_ROWS;
+        const int nst = dual ? 2 * ngrp : ngrp;
+        for (int ph = 0; ph < pl.nph; ++ph) {
+            const int p0 = ph * pl.plen, len = min(pl.plen, K - p0);
+            const int nsteps = len / 16;
+            // ---- B fragments of this warp's k slice, kept in registers for every row group of the phase
+            // (every load is issued before any is used: steps past the end of the phase and rows >= M re-read valid
+            // data and are zeroed afterwards)
+            unsigned fr[NS][FR];
+            {
+                const int last = nsteps - 1 - warp * NS;         // last valid step of this warp (< 0: none)
+                const unsigned char* pbase = xlane + (size_t)(p0 / 16) * 64;
+#pragma unroll
+                for (int s = 0; s < NS; ++s) {
+                    const unsigned char* px = pbase + (size_t)max(min(s, last), -warp * NS) * 64;
+                    if (V == 4) {
+                        const uint2 v = __ldcg(reinterpret_cast<const uint2*>(xrow < M ? px : px - (size_t)xrow * a.ldpk));
+                        fr[s][0] = v.x; fr[s][1] = v.y;
+                    } else {
+#pragma unroll
+                        for (int n = 0; n < NACC; ++n) {
+                            const int row = xrow + 8 * n;
+                            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(row < M ? px + (size_t)(8 * n) * a.ldpk : px - (size_t)xrow * a.ldpk));
+                            fr[s][4 * n + 0] = v.x; fr[s][4 * n + 1] = v.y; fr[s][4 * n + 2] = v.z; fr[s][4 * n + 3] = v.w;
+                        }
+                    }
+                }
+                if (pre_pending) { pre_pending = false; epilogue_prefetch(); }
+#pragma unroll
+                for (int s = 0; s < NS; ++s) {
+                    const bool sv = s <= last;
+                    if (V == 4) {
+                        if (!(sv && xrow < M)) { fr[s][0] = 0u; fr[s][1] = 0u; }
+                    } else {
+#pragma unroll
+                        for (int n = 0; n < NACC; ++n)
+                            if (!(sv && xrow + 8 * n < M)) { fr[s][4 * n + 0] = 0u; fr[s][4 * n + 1] = 0u; fr[s][4 * n + 2] = 0u; fr[s][4 * n + 3] = 0u; }
+                    }
+                }
+            }
+            KG_PROBE(11);
+            // ---- the row groups of this phase, two stages (16 weight rows) at a time
+            const uint32_t a_lane = (uint32_t)((lane & 7) * ST_ROW_BYTES + (warp * NS * 16 + (lane >> 4) * 8) * 2);
+            for (int si = 0; si < nst; si += 2) {
+                const bool two = si + 1 < nst;
+                const int slot_a = slot;
+                const int slot_b = two ? (slot_a + 1 == RING ? 0 : slot_a + 1) : slot_a;
+                const unsigned phase_b = (two && slot_a + 1 == RING) ? phase ^ 1u : phase;
+                float acc[4][4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f; }
+                if (ok) ok = mbar_wait(c, &ctl->full[slot_a], phase, 41);
+                if (ok && two) ok = mbar_wait(c, &ctl->full[slot_b], phase_b, 41);
+                KG_PROBE(12);
+                if (ok) {
+                    // ldmatrix x4: matrices 0, 2 = rows 0-7 (first stage), 1, 3 = rows 8-15 (second stage); k halves 0-7 | 8-15
+                    const uint32_t a_base = smem_u32(ring + (size_t)((lane & 8) ? slot_b : slot_a) * SLOT_BYTES) + a_lane;
+#pragma unroll
+                    for (int s = 0; s < NS; ++s) {
+                        if (warp * NS + s < nsteps) {
+                            unsigned af[4];
+                            ldmatrix_x4(af, a_base + (uint32_t)s * 32u);
+                            if (V == 4) {
+                                mma_bf16_16816(acc[s & 3], af, fr[s][0], fr[s][1]);
+                            } else if (V == 8) {
+                                mma_bf16_16816(acc[(s & 1) * 2], af, fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[(s & 1) * 2 + 1], af, fr[s][2], fr[s][3]);
+                            } else {
+                                mma_bf16_16816(acc[0], af, fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[1], af, fr[s][2], fr[s][3]);
+                                mma_bf16_16816(acc[2], af, fr[s][FR - 4], fr[s][FR - 3]);
+                                mma_bf16_16816(acc[3], af, fr[s][FR - 2], fr[s][FR - 1]);
                             }
                         }
                     }
-                    if (ok) umma_commit(&ctl->bfree[buf]);
                 }
-                if (ok) umma_commit(&ctl->done);
-                c.slot = slot; c.phase = phase;
-            }
-            __syncwarp();
-        } else {
-            // ---- loaders: phase ph of the packed activation rows -> buffer (bph + ph) % NB, as the swizzled B tile
-            const int lt = tid - 32;
-            const int half_n = pl.N >> 1;
-            for (int ph = 0; ph < pl.nph; ++ph) {
-                const int a0 = ph * pl.PA, na = min(pl.natoms - a0, pl.PA);
-                const unsigned gph = bph + (unsigned)ph;
-                const int buf = (int)(gph % NB);
-                const unsigned use = gph / NB;
-                if (use > 0 && ok) ok = mbar_wait(c, &ctl->bfree[buf], (use - 1u) & 1u, 45);
-                if (ok) {
-                    const uint32_t bbase = bbuf + (uint32_t)buf * BBUF_BYTES;
-                    const int total = M * 2 * na * 8;                       // 16-byte pieces: (plane, row, atom, piece)
-                    for (int i = lt; i < total; i += NLOAD) {
-                        const int c8 = i & 7, al = (i >> 3) % na, pm = (i >> 3) / na;
-                        const int p = pm / M, m = pm - p * M;
-                        const int n = p * half_n + m;
-                        const int k0 = (a0 + al) * 64 + c8 * 8;
-                        const uint32_t dst = bbase + (uint32_t)(al * pl.N * 128 + n * 128 + ((c8 ^ (n & 7)) << 4));
-                        if (k0 < K) cp_async16(dst, a.xpk + (size_t)m * a.ldpk + (size_t)p * K * 2 + (size_t)k0 * 2);
-                        else asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
-                    }
+                __syncwarp();
+                KG_PROBE(13);
+                if (ok && lane == 0) { mbar_arrive(&ctl->empty[slot_a]); if (two) mbar_arrive(&ctl->empty[slot_b]); }
+                slot = slot_b; phase = phase_b;
+                if (++slot == RING) { slot = 0; phase ^= 1u; }
+                // ---- add the k-slices in warp order into the row accumulators
+                if (V == 16) cta_sync();                     // single partial-sum buffer: the previous pair's sums have been read
+                float* r = red + (size_t)(V == 16 ? 0 : buf) * NWARPS * 128 + (size_t)warp * NACC * 128;
+                if (V == 16) {
+                    // acc[0] / acc[1]: hi / lo of columns 0-7; acc[2] / acc[3]: hi / lo of columns 8-15
+                    *reinterpret_cast<float2*>(r + g * 8 + 2 * t) = make_float2(acc[0][0] + acc[1][0], acc[0][1] + acc[1][1]);
+                    *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) = make_float2(acc[0][2] + acc[1][2], acc[0][3] + acc[1][3]);
+                    *reinterpret_cast<float2*>(r + 128 + g * 8 + 2 * t) = make_float2(acc[2][0] + acc[3][0], acc[2][1] + acc[3][1]);
+                    *reinterpret_cast<float2*>(r + 128 + (g + 8) * 8 + 2 * t) = make_float2(acc[2][2] + acc[3][2], acc[2][3] + acc[3][3]);
+                } else {
+                    *reinterpret_cast<float2*>(r + g * 8 + 2 * t) =
+                        make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
+                    *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) =
+                        make_float2((acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]), (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]));
                 }
-                if (first && ph == 0) {
-                    // fetched early, used in the epilogue: residual values and output gains of the first superchunk
-                    if (prefetched && a.epi != EPI_HEAD) {
-                        if (a.epi == EPI_RESID)
-                            for (int i = lt; i < M * nu0; i += NLOAD) cp_async4(wk + LW_PRES + (i / nu0) * PRE_NU + i % nu0, a.resid + (size_t)(i / nu0) * a.ldr + pl.u0 + i % nu0);
+                cta_sync();
+                {
+                    // element (weight row r16, activation row m) of the pair; for M <= 8 every thread adds a share of the
+                    // eight k-slices and a fixed butterfly joins the shares, so that no warp lags behind the others
+                    if (V == 16) {
+                        const int r16 = tid >> 4, m = tid & 15;
+                        const float* rb = red + (m >> 3) * 128 + r16 * 8 + (m & 7);
+                        float v = 0.f;
 #pragma unroll
-                        for (int q = 0; q < 2; ++q)
-                            if (a.pk[q].ptr && a.pk[q].gain)
-                                for (int i = lt; i < nu0; i += NLOAD) cp_async4(wk + LW_PREG + q * PRE_NU + i, a.pk[q].gain + pl.u0 + i);
-                    }
-                }
-                cp_async_commit();
-                if (first && ph == 0 && a.ssq_in) {
-                    // thread (m, j) adds the partial sums of CTAs j, j + 14, ... of input row m
-                    const int m = lt / 14, j = lt - m * 14;
-                    float part = 0.f;
-                    if (m < M) for (int q = j; q < nctas; q += 14) part += ldcg_f(a.ssq_in + (size_t)m * nctas + q);
-                    wk[LW_RSP + m * 16 + j] = part;
-                }
-                if (ph >= B_AHEAD) {
-                    cp_async_wait<B_AHEAD>();
-                    fence_proxy_async();
-                    mbar_arrive(&ctl->bready[(gph - B_AHEAD) % NB]);
-                }
-            }
-            cp_async_wait<0>();
-            fence_proxy_async();
-            for (int ph = max(0, pl.nph - B_AHEAD); ph < pl.nph; ++ph) mbar_arrive(&ctl->bready[(bph + (unsigned)ph) % NB]);
-        }
-        bph += (unsigned)pl.nph;
-
-        // ---- accumulators: tensor memory -> shared memory
-        if (ok) ok = mbar_wait(c, &ctl->done, done_cnt & 1u, 43);
-        done_cnt++;
-        tc_fence_after();
-        KG_PROBE(14);
-        {
-            // warp (q, h): lanes 32 q .. 32 q + 31 of the tile, accumulators [h G / 2, (h + 1) G / 2); the two halves are
-            // written ACC2_ROWS apart and added by the epilogue
-            const int q = warp & 3, h = warp >> 2;
-            const int ng = min(pl.G, (K + 15) >> 4);                         // accumulators that received an MMA
-            const int cols_half = pl.G * pl.N / 2;
-            for (int w = 0; w < pl.wtiles; ++w) {
-                const int rows = nu;                                         // one unit tile per superchunk
-                if (32 * q >= rows) continue;                                // the same in every lane of the warp
-                const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(w * pl.G * pl.N + h * cols_half);
-                float o[16];
-#pragma unroll
-                for (int m = 0; m < 16; ++m) o[m] = 0.f;
-                for (int b = 0; b < cols_half; b += 64) {
-                    float v[64];
-                    tmem_ld64(taddr + (uint32_t)b, v);
-                    const int g0 = (h * cols_half + b) / pl.N;
-                    if (pl.N == 16) {
-#pragma unroll
-                        for (int a4 = 0; a4 < 4; ++a4)
-                            if (g0 + a4 < ng) {
-#pragma unroll
-                                for (int m = 0; m < 8; ++m) o[m] += v[16 * a4 + m] + v[16 * a4 + 8 + m];
-                            }
+                        for (int w = 0; w < NWARPS; ++w) v += rb[w * NACC * 128];
+                        float* dst = acc_s + (size_t)((si >> 1) * 16 + r16) * MP + m;
+                        *dst = ph == 0 ? v : *dst + v;
                     } else {
+                        constexpr int TPE = V == 4 ? 4 : 2;                  // threads per element
+                        constexpr int WPT = NWARPS / TPE;                    // k-slices per thread
+                        const int e = tid / TPE, q = tid % TPE;
+                        const int r16 = V == 4 ? e >> 2 : e >> 3;
+                        const int m = V == 4 ? e & 3 : e & 7;
+                        const float* rb = red + (size_t)buf * NWARPS * 128 + r16 * 8 + m;
+                        float v = 0.f;
 #pragma unroll
-                        for (int a2 = 0; a2 < 2; ++a2)
-                            if (g0 + a2 < ng) {
+                        for (int w = 0; w < WPT; ++w) v += V == 4 ? rb[(q * WPT + w) * 128] + rb[(q * WPT + w) * 128 + 4] : rb[(q * WPT + w) * 128];
 #pragma unroll
-                                for (int m = 0; m < 16; ++m) o[m] += v[32 * a2 + m] + v[32 * a2 + 16 + m];
-                            }
+                        for (int o = 1; o < TPE; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (q == 0) {
+                            float* dst = acc_s + (size_t)((si >> 1) * 16 + r16) * MP + m;
+                            *dst = ph == 0 ? v : *dst + v;
+                        }
                     }
                 }
-                const int i = 32 * q + lane;
-                if (i < rows) {
-                    const int arow = (dual ? ((i >> 3) * 16 + (i & 7) + 8 * w) : i) + h * ACC2_ROWS;
-                    float4* dst = reinterpret_cast<float4*>(acc_s + (size_t)arow * MP);
-                    dst[0] = make_float4(o[0], o[1], o[2], o[3]);
-                    dst[1] = make_float4(o[4], o[5], o[6], o[7]);
-                    if (pl.N == 32) { dst[2] = make_float4(o[8], o[9], o[10], o[11]); dst[3] = make_float4(o[12], o[13], o[14], o[15]); }
-                }
+                KG_PROBE(14);
+                buf ^= 1;
             }
         }
-        tc_fence_before();
-
         // ---- epilogue of this superchunk
-        if (first) {
-            cp_async_wait<0>();
+        if (sc0 == pl.u0) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
             cta_sync();
             if (tid < M_MAX) {
                 float r = 1.0f;
                 if (a.ssq_in && tid < M) {
                     float ss = 0.f;
-                    for (int j = 0; j < 14; ++j) ss += wk[LW_RSP + tid * 16 + j];
+                    for (int j = 0; j < 16; ++j) ss += wk[LW_RSP + tid * 16 + j];
                     r = rsqrtf(ss / (float)K + a.eps);
                 }
                 rs[tid] = r;
@@ -861,7 +769,7 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                     const float f = rs[m] * a.scale;
                     float zm = -INFINITY; int im = 0x7fffffff;
                     for (int r = lane; r < nu; r += 32) {
-                        const float z = (acc_s[(size_t)r * MP + m] + acc_s[(size_t)(ACC2_ROWS + r) * MP + m]) * f;
+                        const float z = acc_s[(size_t)r * MP + m] * f;
                         if (a.logits_dbg) a.logits_dbg[(size_t)m * a.ld_dbg + sc0 + r] = z;
                         if (arg_better(z, sc0 + r, zm, im)) { zm = z; im = sc0 + r; }
                     }
@@ -872,16 +780,15 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                         if (arg_better(z2, i2, zm, im)) { zm = z2; im = i2; }
                     }
                     float e = 0.f;
-                    for (int r = lane; r < nu; r += 32) e += expf((acc_s[(size_t)r * MP + m] + acc_s[(size_t)(ACC2_ROWS + r) * MP + m]) * f - zm);
+                    for (int r = lane; r < nu; r += 32) e += expf(acc_s[(size_t)r * MP + m] * f - zm);
                     e = warp_sum(e);
                     if (nu > 0) head_merge(hs[q], zm, e, im);
                 }
             }
         } else {
-            emit_rows(a, acc_s, ACC2_ROWS * MP, wk, sc0, nu, prefetched && first, ssq_acc);
+            emit_rows(a, wk, sc0, nu, prefetched && sc0 == pl.u0, ssq_acc);
         }
-        first = false;
-        cta_sync();                                  // the B buffers / tensor memory are rewritten by the next superchunk / operator
+        cta_sync();                                  // acc_s is rewritten by the next superchunk / operator
         KG_PROBE(15);
     }
     if (a.epi == EPI_HEAD && lane == 0) {
@@ -892,7 +799,7 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
         }
     }
     if (a.epi != EPI_HEAD && a.ssq_out && tid < M) a.ssq_out[(size_t)tid * nctas + cta] = ssq_acc;
-    if (tid == 0) { c.bph = bph; c.done_cnt = done_cnt; }
+    c.slot = slot; c.phase = phase;
 }
 
 // Rows that do not come out of a linear operator (token embeddings): every CTA takes its slice of
@@ -902,21 +809,19 @@ template <typename F>
 __device__ __forceinline__ void emit_plain_rows(LinArgs& a, Ctx& c, F value) {
     const int tid = threadIdx.x;
     float* wk = reinterpret_cast<float*>(c.smem + WORK_OFF);
-    float* acc_s = reinterpret_cast<float*>(c.smem + BBUF_OFF);
     const int u0 = (int)((unsigned)a.N * (unsigned)c.cta / (unsigned)c.nctas);
     const int u1 = (int)((unsigned)a.N * (unsigned)(c.cta + 1) / (unsigned)c.nctas);
     float ssq_acc = 0.f;
     a.epi = EPI_STORE;
     if (tid < M_MAX) wk[LW_RS + tid] = 1.0f;
-    for (int sc0 = u0; sc0 < u1; sc0 += ACC2_ROWS) {
-        const int nu = min(ACC2_ROWS, u1 - sc0);
+    for (int sc0 = u0; sc0 < u1; sc0 += SC_ROWS) {
+        const int nu = min(SC_ROWS, u1 - sc0);
         for (int idx = tid; idx < nu * a.M; idx += NTHREADS) {
             const int r = idx % nu, m = idx / nu;
-            acc_s[(size_t)r * MP + m] = value(m, sc0 + r);
-            acc_s[(size_t)(ACC2_ROWS + r) * MP + m] = 0.f;
+            wk[LW_ACC + (size_t)r * MP + m] = value(m, sc0 + r);
         }
         cta_sync();
-        emit_rows(a, acc_s, ACC2_ROWS * MP, wk, sc0, nu, false, ssq_acc);
+        emit_rows(a, wk, sc0, nu, false, ssq_acc);
         cta_sync();
     }
     if (a.ssq_out && tid < a.M) a.ssq_out[(size_t)tid * c.nctas + c.cta] = ssq_acc;
@@ -1003,7 +908,7 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
 }
 
 // One linear operator, called by every thread of the CTA; `stream` selects the streamed tensor-core
-// path (bf16 weights; decided once per model so that the packed activation
+// path (bf16 weights, every K a multiple of 16; decided once per model so that the packed activation
 // rows exist wherever they are read).  Consumers return after their part; whether the grid must stop
 // is learnt at the next grid barrier.  The producer returns false when one of its waits gave up.
 template <typename WT>
@@ -1016,7 +921,7 @@ __device__ __forceinline__ bool linear_op(const LinArgs* sa, Ctx& c, bool stream
     }
     if (publish) cta_sync();
     if (stream) {
-        lin_consume(*sa, c);
+        if (sa->M <= 4) lin_consume<4>(*sa, c); else if (sa->M <= 8) lin_consume<8>(*sa, c); else lin_consume<16>(*sa, c);
     } else {
         lin_simple<WT>(*sa, c);
     }
@@ -1238,7 +1143,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
     WT* kc = reinterpret_cast<WT*>(a.kc);
     WT* vc = reinterpret_cast<WT*>(a.vc);
 
-    float* qs = reinterpret_cast<float*>(c.smem + BBUF_OFF);       // [M_MAX][HD_MAX]
+    float* qs = reinterpret_cast<float*>(c.smem + WORK_OFF);       // [M_MAX][HD_MAX]
     float* mb = qs + M_MAX * HD_MAX;                               // [NWARPS][ATT_RB][ATT_MB_STRIDE]
     float* pbuf = mb + NWARPS * ATT_RB * ATT_MB_STRIDE + warp * 40;      // [NWARPS][40] probabilities of a key group
     KG_PROBE(20);
@@ -1308,7 +1213,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                 if (S == 1) {
                     const float ov = num / den;
                     a.out[(size_t)i * d + hh * hd + e] = ov;
-                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, d, hh * hd + e, ov);
+                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
                 } else {
                     D.att_po[(((size_t)i * H + hh) * S_CAP + s) * hd + e] = num;
                     if (e == 0) {
@@ -1346,7 +1251,7 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                     }
                     const float ov = num / den;
                     a.out[(size_t)i * d + hh * hd + e] = ov;
-                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, d, hh * hd + e, ov);
+                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
                 }
             }
             cta_sync();
@@ -1362,6 +1267,6 @@ __device__ __forceinline__ void attention_op(const Dev& D, const AttArgs* sa, Ct
     else attention_impl<WT, 1>(D, *sa, c);
 }
 
-static_assert((M_MAX * HD_MAX + NWARPS * ATT_RB * ATT_MB_STRIDE + NWARPS * 40) * 4 <= NB * BBUF_BYTES + WORK_BYTES, "attention buffers do not fit in the work area");
+static_assert((M_MAX * HD_MAX + NWARPS * ATT_RB * ATT_MB_STRIDE + NWARPS * 40) * 4 <= WORK_BYTES, "attention buffers do not fit in the work area");
 
 }  // namespace kg

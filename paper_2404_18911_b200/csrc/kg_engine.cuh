@@ -54,7 +54,7 @@ struct Engine {
     __device__ size_t cache_layer_stride() const {
         return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
     }
-    __device__ __forceinline__ size_t ldpk() const { return (size_t)D.dm.d * 4; }       // bytes of a packed row of d elements
+    __device__ __forceinline__ size_t ldpk() const { return (size_t)D.dm.d * 4; }
     __device__ __forceinline__ ActIn act_h() const { return ActIn{D.h, D.hA_pk, D.ssq_hA}; }
     // the residual stream as an output, packed for a reader whose norm gain is `gain`
     __device__ __forceinline__ ActOut out_h(const float* gain) const {
@@ -93,7 +93,7 @@ struct Engine {
         LinArgs& q = t->lin[0];
         q = LinArgs{};
         q.M = M; q.eps = dm.eps;
-        q.W = lw.wqkv; q.tmW = lw.tm_qkv; q.tm_global = 1; q.N = 3 * dm.d; q.K = dm.d;
+        q.W = lw.wqkv; q.N = 3 * dm.d; q.K = dm.d;
         q.x = in.x; q.ldx = dm.d; q.gain = lw.g1; q.xpk = in.pk; q.ldpk = (int)ldpk(); q.ssq_in = in.ssq;
         q.epi = EPI_STORE; q.out = D.qkv; q.ldo = 3 * dm.d;
         AttArgs& at = t->att;
@@ -104,7 +104,7 @@ struct Engine {
         LinArgs& o = t->lin[1];
         o = LinArgs{};
         o.M = M; o.eps = dm.eps;
-        o.W = lw.wo; o.tmW = lw.tm_o; o.tm_global = 1; o.N = dm.d; o.K = dm.d; o.x = D.attn; o.ldx = dm.d;
+        o.W = lw.wo; o.N = dm.d; o.K = dm.d; o.x = D.attn; o.ldx = dm.d;
         o.xpk = D.attn_pk; o.ldpk = (int)ldpk();
         o.epi = EPI_RESID; o.resid = in.x; o.ldr = dm.d; o.out = o_out; o.ldo = dm.d;
         o.pk[0] = o_pk; o.ldpk_out = (int)ldpk(); o.ssq_out = o_ssq;
@@ -121,14 +121,14 @@ struct Engine {
             LinArgs& gu = t->lin[2];
             gu = LinArgs{};
             gu.M = M; gu.eps = dm.eps;
-            gu.W = lw.wgate; gu.W2 = lw.wup; gu.tmW = lw.tm_gate; gu.tmW2 = lw.tm_up; gu.tm_global = 1; gu.N = dm.F; gu.K = dm.d; gu.x = D.h; gu.ldx = dm.d; gu.gain = lw.g2;
+            gu.W = lw.wgate; gu.W2 = lw.wup; gu.N = dm.F; gu.K = dm.d; gu.x = D.h; gu.ldx = dm.d; gu.gain = lw.g2;
             gu.xpk = D.hB_pk; gu.ldpk = (int)ldpk(); gu.ssq_in = D.ssq_hB;
             gu.epi = EPI_SWIGLU; gu.out = D.act; gu.ldo = dm.F;
             gu.pk[0] = PkOut{nullptr, D.act_pk}; gu.ldpk_out = dm.F * 4;
             LinArgs& dn = t->lin[3];
             dn = LinArgs{};
             dn.M = M; dn.eps = dm.eps;
-            dn.W = lw.wdown; dn.tmW = lw.tm_down; dn.tm_global = 1; dn.N = dm.d; dn.K = dm.F; dn.x = D.act; dn.ldx = dm.F;
+            dn.W = lw.wdown; dn.N = dm.d; dn.K = dm.F; dn.x = D.act; dn.ldx = dm.F;
             dn.xpk = D.act_pk; dn.ldpk = dm.F * 4;
             dn.epi = EPI_RESID; dn.resid = D.h; dn.ldr = dm.d; dn.out = out.x; dn.ldo = dm.d;
             dn.pk[0] = out.pk[0]; dn.pk[1] = out.pk[1]; dn.ldpk_out = (int)ldpk(); dn.ssq_out = out.ssq;
@@ -175,7 +175,7 @@ struct Engine {
             LinArgs& a = t->lin[0];
             a = LinArgs{};
             a.M = M; a.eps = dm.eps;
-            a.W = D.head; a.tmW = D.tm_head; a.tm_global = 1; a.N = dm.V; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = gain;
+            a.W = D.head; a.N = dm.V; a.K = dm.d; a.x = in.x; a.ldx = dm.d; a.gain = gain;
             a.xpk = in.pk; a.ldpk = (int)ldpk(); a.ssq_in = in.ssq;
             a.epi = EPI_HEAD; a.scale = dm.logit_scale; a.head_part = D.head_part;
             a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
@@ -385,12 +385,10 @@ struct Engine {
 
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
-    extern __shared__ __align__(1024) char smem[];
-    const bool tc = D.dm.stream != 0;
-    Ctx& c = ctx_init(smem, D.st, D.bar, true, tc);
+    extern __shared__ __align__(128) char smem[];
+    Ctx& c = ctx_init(smem, D.st, D.bar, true);
     Engine<WT> eng(D, c, pg);
     eng.run();
-    ctx_fini(c, tc);
 }
 
 }  // namespace kg
