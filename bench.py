@@ -31,9 +31,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the decode launch, from the ncu
-# capture summarised in profiles/kg_persistent_kernel_7b-4layers_decode.md (a 4-layer case of the same kernel; the
-# traffic is weights + KV and grows in proportion to the bytes a launch streams).  Set to None when the kernel changes.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the decode launch, from an ncu
+# capture of a 4-layer case of the same kernel (the traffic is weights + KV and grows in proportion to the bytes a
+# launch streams).  Set to None when the kernel changes.
 NCU_TRAFFIC_RATIO = 1.016
 
 METRIC = "batch-1 generated tokens/s"
