@@ -176,7 +176,7 @@ def test_api_errors(binding):
     g.verify()
 
 
-def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0, conf_tol=1e-3):
+def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0, conf_tol=1e-3, eta=None, gamma=None):
     """Full-size shape, short prompt: a handful of lock-step rounds against the fp32 oracle (the oracle's
     weights for these shapes only fit in fp32, and a full-length prompt would take it hours)."""
     from parity_harness import lockstep
@@ -184,10 +184,12 @@ def _sampled_big_shape(binding, name, n_prompt, n_new, rounds_mode=0, conf_tol=1
     g = binding.KangarooModel(shape, debug_logits=True)
     o = ko.KangarooOracle(shape, ki.make_weights(shape), np.float64 if name == "7b" else np.float32)
     prompt = ki.make_prompt(shape, n_prompt).tolist()
-    res = lockstep(g, o, prompt, n_new, shape.eta, shape.gamma, rounds_mode, conf_tol=conf_tol)
+    eta = shape.eta if eta is None else eta
+    gamma = shape.gamma if gamma is None else gamma
+    res = lockstep(g, o, prompt, n_new, eta, gamma, rounds_mode, conf_tol=conf_tol)
     assert len(res["flips"]) <= 1, res["flips"]
     assert res["max_logit_err"] < 2e-2 and res["max_conf_err"] < conf_tol, res
-    assert all(1 <= s <= shape.gamma + 1 for s in res["S"])
+    assert all(1 <= s <= gamma + 1 for s in res["S"])
     return res
 
 
@@ -196,6 +198,14 @@ def test_7b_shape_sampled_rounds(binding):
     target tokens, accept lengths and logits against the oracle."""
     res = _sampled_big_shape(binding, "7b", 24, 12)
     assert len(res["tokens"]) >= 12
+
+
+def test_7b_shape_fixed_step_drafting_rounds(binding):
+    """The same model with eta = 0 (Section 4.3's fixed-step drafting: every round drafts gamma tokens, so the verify
+    pass runs on gamma + 1 = 7 rows, the wider of the small-M tensor-core variants) in the stop mode that drops the
+    low-confidence token: drafts, confidences, target tokens, accept lengths and logits against the oracle."""
+    res = _sampled_big_shape(binding, "7b", 20, 14, rounds_mode=1, eta=0.0, gamma=6)
+    assert len(res["tokens"]) >= 14
 
 
 @pytest.mark.parametrize("name", ["13b", "33b"])
