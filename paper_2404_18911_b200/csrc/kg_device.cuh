@@ -939,6 +939,27 @@ __device__ __forceinline__ void head_final(const float4* part, int nctas, int m,
     p = 1.0f / tot.sum;
 }
 
+// The same merge by a whole warp: every lane merges the partials of CTAs lane, lane + 32, ... (independent loads, one
+// round trip instead of one per CTA), then a butterfly of merges leaves the identical total in every lane (the merge
+// of two partials is the same whichever of the two lanes computes it).
+__device__ __forceinline__ void head_final_warp(const float4* part, int nctas, int m, int& tok, float& p) {
+    const int lane = threadIdx.x & 31;
+    HeadStat tot; tot.zmax = 0.f; tot.sum = 0.f; tot.arg = 0;
+    for (int cta = lane; cta < nctas; cta += 32) {
+        const float4 v = __ldcg(part + (size_t)cta * M_MAX + m);
+        head_merge(tot, v.x, v.y, __float_as_int(v.z));
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float z = __shfl_xor_sync(0xffffffffu, tot.zmax, o);
+        const float sm = __shfl_xor_sync(0xffffffffu, tot.sum, o);
+        const int ar = __shfl_xor_sync(0xffffffffu, tot.arg, o);
+        head_merge(tot, z, sm, ar);
+    }
+    tok = tot.arg;
+    p = 1.0f / tot.sum;
+}
+
 // ------------------------------------------------------------------------------------ attention operator
 struct AttArgs {
     const float* qkv;      // [M][3d] raw q, k, v rows of this pass
@@ -1238,16 +1259,28 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
             if (*(volatile int*)&c.ctl->att_last) {
                 for (int idx = tid; idx < M * hd; idx += NTHREADS) {
                     const int i = idx / hd, e = idx % hd;
-                    const float* ml = D.att_ml + ((size_t)i * H + hh) * S_CAP * 2;
+                    // every load of a pass is issued before any is used: two round trips, not two per split
+                    const float2* ml = reinterpret_cast<const float2*>(D.att_ml + ((size_t)i * H + hh) * S_CAP * 2);
+                    const float* po = D.att_po + ((size_t)i * H + hh) * S_CAP * hd + e;
+                    float2 mlv[S_CAP];
+                    float pov[S_CAP];
+#pragma unroll
+                    for (int q = 0; q < S_CAP; ++q) {
+                        const int qq = q < S ? q : 0;
+                        mlv[q] = __ldcg(ml + qq);
+                        pov[q] = ldcg_f(po + (size_t)qq * hd);
+                    }
                     float mx = -INFINITY;
-                    for (int q = 0; q < S; ++q) mx = fmaxf(mx, ldcg_f(ml + q * 2));
+#pragma unroll
+                    for (int q = 0; q < S_CAP; ++q) if (q < S) mx = fmaxf(mx, mlv[q].x);
                     float den = 0.f, num = 0.f;
-                    for (int q = 0; q < S; ++q) {
-                        const float mq = ldcg_f(ml + q * 2);
-                        if (mq == -INFINITY) continue;
-                        const float w = ex2f(mq - mx);
-                        den += ldcg_f(ml + q * 2 + 1) * w;
-                        num += ldcg_f(D.att_po + (((size_t)i * H + hh) * S_CAP + q) * hd + e) * w;
+#pragma unroll
+                    for (int q = 0; q < S_CAP; ++q) {
+                        if (q < S && mlv[q].x != -INFINITY) {
+                            const float w = ex2f(mlv[q].x - mx);
+                            den += mlv[q].y * w;
+                            num += pov[q] * w;
+                        }
                     }
                     const float ov = num / den;
                     a.out[(size_t)i * d + hh * hd + e] = ov;

@@ -192,10 +192,10 @@ struct Engine {
             if (!ok) return false;
         } else {
             if (!grid_sync(c, 30)) return false;
-            if (threadIdx.x < M) {
+            for (int m = threadIdx.x >> 5; m < M; m += NWARPS) {           // one warp per row
                 int tk; float p;
-                head_final(D.head_part, c.nctas, threadIdx.x, tk, p);
-                c.ctl->head_tok[threadIdx.x] = tk; c.ctl->head_p[threadIdx.x] = p;
+                head_final_warp(D.head_part, c.nctas, m, tk, p);
+                if ((threadIdx.x & 31) == 0) { c.ctl->head_tok[m] = tk; c.ctl->head_p[m] = p; }
             }
             cta_sync();
             if (threadIdx.x == 0) mbar_arrive(&c.ctl->mail);
