@@ -202,12 +202,16 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsign
                  ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// The top bit of the grid barrier's arrival counter tells every CTA that some wait has given up: they learn it from
+// the word they poll anyway, without a second load.
+constexpr unsigned BAR_ABORT = 0x80000000u;
 __device__ __forceinline__ void record_timeout(Ctx& c, int where) {
     *(volatile int*)&c.ctl->abort = 1;
     if (c.st) {
         atomicCAS(&c.st->status, 0, ST_TIMEOUT);
         c.st->timeout_where = where;
     }
+    if (c.grid && c.bar) atomicOr(c.bar, BAR_ABORT);
 }
 
 // Bounded wait on an mbarrier phase.  Returns false when this CTA has given up (here or elsewhere).
@@ -300,7 +304,8 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
     cta_sync();
     KG_PROBE(1);
     if (threadIdx.x == 0) {
-        // bar[0] counts arrivals (monotonic over the launch): one release-add, then poll until every CTA has arrived
+        // bar[0] counts arrivals (monotonic over the launch, far below 2^31): one release-add, then poll until every CTA
+        // has arrived or the abort bit appears
         c.bar_target += (unsigned)c.nctas;
         const unsigned gen = c.bar_target;
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.bar) : "memory");
@@ -308,14 +313,15 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
         {
             const long long t0 = clock64();
             unsigned spins = 0;
-            while ((int)(ld_acquire_u32(c.bar) - gen) < 0) {
+            while (true) {
+                const unsigned v = ld_acquire_u32(c.bar);
+                if (v & BAR_ABORT) { ok = 0; break; }
+                if ((int)(v - gen) >= 0) break;
                 if (((++spins) & 63u) == 0u) {
-                    if (*(volatile int*)&c.st->status != 0) { ok = 0; break; }
                     if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
                 }
             }
         }
-        if (*(volatile int*)&c.st->status != 0) ok = 0;
         if (!ok) *(volatile int*)&c.ctl->abort = 1;          // lets the producer warp leave its waits
         c.ctl->sync_ok = ok;
     }
