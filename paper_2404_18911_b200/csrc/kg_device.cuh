@@ -1178,28 +1178,30 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
     for (int item = c.cta; item < H * S; item += c.nctas) {
         const int hh = item / S, s = item % S;
         const int kb = s * chunk, ke = min(T, kb + chunk);
-        // q rows: RoPE, pre-scaled by 1/sqrt(hd)
+        // q rows: RoPE, pre-scaled by 1/sqrt(hd) (loads first: the angle arithmetic runs while they are in flight)
         for (int idx = tid; idx < M * half; idx += NTHREADS) {
             const int i = idx / half, e = idx % half;
-            float cs, sn; rope_cs(D, pos0 + i, e, cs, sn);
             const float x1 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * hd + e);
             const float x2 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * hd + e + half);
+            float cs, sn; rope_cs(D, pos0 + i, e, cs, sn);
             qs[i * HD_MAX + e] = (x1 * cs - x2 * sn) * sc;
             qs[i * HD_MAX + e + half] = (x2 * cs + x1 * sn) * sc;
         }
-        // append this pass's K / V rows that fall into my key range
+        // append this pass's K / V rows that fall into my key range (every load of an element before its first use)
         {
             const int nb = max(kb, pos0), ne = ke;
             for (int idx = tid; idx < (ne - nb) * half; idx += NTHREADS) {
                 const int pos = nb + idx / half, e = idx % half, i = pos - pos0;
-                float cs, sn; rope_cs(D, pos, e, cs, sn);
                 const float* src = a.qkv + (size_t)i * 3 * d + hh * hd;
                 const float k1 = ldcg_f(src + d + e), k2 = ldcg_f(src + d + e + half);
-                const size_t base = (((size_t)D.page_table[pos >> D.dm.ps_shift] * H + hh) * ps + (pos & (ps - 1))) * hd;
+                const float v1 = ldcg_f(src + 2 * d + e), v2 = ldcg_f(src + 2 * d + e + half);
+                const int page = __ldg(D.page_table + (pos >> D.dm.ps_shift));
+                float cs, sn; rope_cs(D, pos, e, cs, sn);
+                const size_t base = (((size_t)page * H + hh) * ps + (pos & (ps - 1))) * hd;
                 kc[base + e] = float_to_wt<WT>(k1 * cs - k2 * sn);
                 kc[base + e + half] = float_to_wt<WT>(k2 * cs + k1 * sn);
-                vc[base + e] = float_to_wt<WT>(ldcg_f(src + 2 * d + e));
-                vc[base + e + half] = float_to_wt<WT>(ldcg_f(src + 2 * d + e + half));
+                vc[base + e] = float_to_wt<WT>(v1);
+                vc[base + e + half] = float_to_wt<WT>(v2);
             }
         }
         cta_sync();
