@@ -1145,6 +1145,54 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
     }
 }
 
+// The last split of a head to arrive merges the S partial (max, sum, o) of every row in split order.  SC >= S is the
+// compile-time bound of the split loop; U elements per thread are handled together, and every load of such a batch is
+// issued before any is used, so that a batch costs one L2 round trip.
+template <int SC, int U>
+__device__ __forceinline__ void att_merge_splits(const Dev& D, const AttArgs& a, int hh, int S, int M) {
+    const int tid = threadIdx.x, H = D.dm.H, hd = D.dm.hd, d = D.dm.d;
+    const int total = M * hd;
+    for (int idx0 = tid; idx0 < total; idx0 += NTHREADS * U) {
+        float2 mlv[U][SC];
+        float pov[U][SC];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = idx0 + u * NTHREADS < total ? idx0 + u * NTHREADS : idx0;
+            const int i = idx / hd, e = idx % hd;
+            const float2* ml = reinterpret_cast<const float2*>(D.att_ml + ((size_t)i * H + hh) * S_CAP * 2);
+            const float* po = D.att_po + ((size_t)i * H + hh) * S_CAP * hd + e;
+#pragma unroll
+            for (int q = 0; q < SC; ++q) {
+                const int qq = q < S ? q : 0;
+                mlv[u][q] = __ldcg(ml + qq);
+                pov[u][q] = ldcg_f(po + (size_t)qq * hd);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = idx0 + u * NTHREADS;
+            if (idx < total) {
+                const int i = idx / hd, e = idx % hd;
+                float mx = -INFINITY;
+#pragma unroll
+                for (int q = 0; q < SC; ++q) if (q < S) mx = fmaxf(mx, mlv[u][q].x);
+                float den = 0.f, num = 0.f;
+#pragma unroll
+                for (int q = 0; q < SC; ++q) {
+                    if (q < S && mlv[u][q].x != -INFINITY) {
+                        const float w = ex2f(mlv[u][q].x - mx);
+                        den += mlv[u][q].y * w;
+                        num += pov[u][q] * w;
+                    }
+                }
+                const float ov = num / den;
+                a.out[(size_t)i * d + hh * hd + e] = ov;
+                if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
+            }
+        }
+    }
+}
+
 template <typename WT, int DPL>
 __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx& c) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1265,35 +1313,9 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
             }
             cta_sync();
             if (*(volatile int*)&c.ctl->att_last) {
-                for (int idx = tid; idx < M * hd; idx += NTHREADS) {
-                    const int i = idx / hd, e = idx % hd;
-                    // every load of a pass is issued before any is used: two round trips, not two per split
-                    const float2* ml = reinterpret_cast<const float2*>(D.att_ml + ((size_t)i * H + hh) * S_CAP * 2);
-                    const float* po = D.att_po + ((size_t)i * H + hh) * S_CAP * hd + e;
-                    float2 mlv[S_CAP];
-                    float pov[S_CAP];
-#pragma unroll
-                    for (int q = 0; q < S_CAP; ++q) {
-                        const int qq = q < S ? q : 0;
-                        mlv[q] = __ldcg(ml + qq);
-                        pov[q] = ldcg_f(po + (size_t)qq * hd);
-                    }
-                    float mx = -INFINITY;
-#pragma unroll
-                    for (int q = 0; q < S_CAP; ++q) if (q < S) mx = fmaxf(mx, mlv[q].x);
-                    float den = 0.f, num = 0.f;
-#pragma unroll
-                    for (int q = 0; q < S_CAP; ++q) {
-                        if (q < S && mlv[q].x != -INFINITY) {
-                            const float w = ex2f(mlv[q].x - mx);
-                            den += mlv[q].y * w;
-                            num += pov[q] * w;
-                        }
-                    }
-                    const float ov = num / den;
-                    a.out[(size_t)i * d + hh * hd + e] = ov;
-                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * hd + e, ov);
-                }
+                if (S <= 4) att_merge_splits<4, 4>(D, a, hh, S, M);
+                else if (S <= 8) att_merge_splits<8, 2>(D, a, hh, S, M);
+                else att_merge_splits<S_CAP, 1>(D, a, hh, S, M);
             }
             cta_sync();
         }
