@@ -6,7 +6,8 @@ rule): only a counter-based pseudo-random generator, the five workload shapes, a
 tensor naming that says which counter stream fills which tensor.
 
 The CUDA library carries its own implementation of the same generator so that a 66 GB
-model never has to cross PCIe; `tests/test_synth_device.py` checks the two bit for bit.
+model never has to cross PCIe; `tests/test_gpu_parity.py::test_device_weights_equal_host_generator`
+checks the two bit for bit.
 """
 from .synth import (  # noqa: F401
     splitmix64,
@@ -19,4 +20,5 @@ from .synth import (  # noqa: F401
     TensorId,
     GAUSS_INT_STD,
 )
-from .configs import KgShape, CONFIGS, get_config, make_weights, make_prompt, param_counts, microbench_state  # noqa: F401
+from .configs import (KgShape, CONFIGS, get_config, make_weights, LazyWeights, make_prompt, param_counts,  # noqa: F401
+                      microbench_state)

@@ -174,3 +174,77 @@ def microbench_state(shape: KgShape, T: int, n_d: int, seed: int) -> dict:
     feat = synth.fill_f32(seed, int(TensorId.HIDDEN), 17 * d, 1.0, False).reshape(17, d)
     toks = synth.uniform_tokens(seed, int(TensorId.DRAFT), 1001, shape.vocab)
     return {"k": k, "v": v, "feat": feat, "x0": int(toks[1000]), "drafts": [int(t) for t in toks[:max(n_d, 0)]]}
+
+
+# ---- weights regenerated on demand ---------------------------------------------------
+
+class _LazyBlock:
+    """One layer's (or the adapter's) tensors, produced when they are read."""
+
+    def __init__(self, owner, layer, names):
+        self._owner, self._layer, self._names = owner, layer, names
+
+    def __getitem__(self, name):
+        return self._owner._get(self._layer, self._names[name])
+
+    def keys(self):
+        return self._names.keys()
+
+
+class LazyWeights:
+    """The same tensors as make_weights, with the same nesting (w["layers"][i]["wqkv"], w["adapter"]["wo"],
+    w["head"], ...), produced from their counter streams when they are read and converted to `dtype`.
+    For shapes whose weights do not fit in host memory at 8 bytes per value.
+
+    The tensors read first are kept until `budget_bytes` are held; every tensor read after that is
+    regenerated on each read into one of two reusable buffers of its shape, so such an array is only valid
+    until the second-next read of a tensor of the same shape (a matrix-vector product uses it at once).
+    `lazy_weights = True` tells a consumer to take the tensors as they come instead of converting the whole
+    collection up front."""
+    lazy_weights = True
+
+    def __init__(self, shape: KgShape, dtype=np.float64, budget_bytes: int = 16 << 30):
+        self.shape, self.dtype, self.budget = shape, np.dtype(dtype), int(budget_bytes)
+        self._held = {}          # (layer, name) -> array kept for good
+        self._bytes = 0
+        self._scratch = {}       # array shape -> [buffers, next buffer]
+        L = shape.n_layers
+        mats = ("wqkv", "wo", "wgate", "wup", "wdown")
+        self._top = {"embed": (None, "embed"), "head": (None, "head"), "g_final": (None, "g_final")}
+        self._layers = [_LazyBlock(self, i, {**{n: n for n in mats}, "g1": "g1", "g2": "g2"}) for i in range(L)]
+        self._adapter = _LazyBlock(self, L, {"wqkv": "wqkv", "wo": "wo", "g_in": "g1", "g_last": "g2"})
+
+    def __getitem__(self, key):
+        if key == "layers":
+            return self._layers
+        if key == "adapter":
+            return self._adapter
+        return self._get(*self._top[key])
+
+    def _make(self, layer, name):
+        s = self.shape
+        if name == "g_final":
+            return gain_vector(s, int(TensorId.GFINAL))
+        if name == "g1":
+            return gain_vector(s, layer_tid(layer, TensorId.G1))
+        if name == "g2":
+            return gain_vector(s, layer_tid(layer, TensorId.G2))
+        return weight_tensor(s, name, layer)
+
+    def _get(self, layer, name):
+        key = (layer, name)
+        a = self._held.get(key)
+        if a is not None:
+            return a
+        src = self._make(layer, name)
+        nbytes = src.size * self.dtype.itemsize
+        if self._bytes + nbytes <= self.budget:
+            a = src.astype(self.dtype)
+            self._held[key] = a
+            self._bytes += nbytes
+            return a
+        slot = self._scratch.setdefault(src.shape, [[np.empty(src.shape, self.dtype), np.empty(src.shape, self.dtype)], 0])
+        a = slot[0][slot[1]]
+        slot[1] ^= 1
+        np.copyto(a, src)
+        return a

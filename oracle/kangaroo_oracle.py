@@ -156,8 +156,8 @@ class KangarooOracle:
         self.reset()
 
     def _cast(self, w):
-        if self.dt == np.float32:
-            return w
+        if self.dt == np.float32 or getattr(w, "lazy_weights", False):
+            return w                  # a lazy collection hands out tensors of the wanted type one at a time
         if isinstance(w, dict):
             return {k: self._cast(v) for k, v in w.items()}
         if isinstance(w, list):

@@ -109,3 +109,26 @@ def test_shapes_match_the_five_configs():
     for s in c.values():
         assert s.n_heads * s.head_dim == s.d_model
         assert s.max_seq >= s.n_prompt + s.n_gen + s.gamma_max + 1
+
+
+def test_lazy_weights_equal_the_eager_recipe():
+    """Tensors regenerated on demand are bit-identical to make_weights, whether they are kept or rebuilt into the
+    reusable buffers (budget 0: nothing is kept)."""
+    shape = ki.get_config("tiny").with_(gain_std=0.1)
+    w = ki.make_weights(shape)
+    for budget in (0, 600_000, 1 << 40):
+        lw = ki.LazyWeights(shape, np.float64, budget)
+        assert getattr(lw, "lazy_weights", False)
+        for i in range(shape.n_layers):
+            for n in ("wqkv", "wo", "wgate", "wup", "wdown", "g1", "g2"):
+                a = lw["layers"][i][n]
+                assert a.dtype == np.float64 and np.array_equal(a, w["layers"][i][n].astype(np.float64)), (budget, i, n)
+        for n in ("wqkv", "wo", "g_in", "g_last"):
+            assert np.array_equal(lw["adapter"][n], w["adapter"][n].astype(np.float64))
+        for n in ("embed", "head", "g_final"):
+            assert np.array_equal(lw[n], w[n].astype(np.float64))
+        assert lw._bytes <= budget
+    # two tensors of one shape read back to back stay valid together (two buffers per shape)
+    lw = ki.LazyWeights(shape, np.float64, 0)
+    g, u = lw["layers"][0]["wgate"], lw["layers"][0]["wup"]
+    assert np.array_equal(g, w["layers"][0]["wgate"]) and np.array_equal(u, w["layers"][0]["wup"])

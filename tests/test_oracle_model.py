@@ -85,7 +85,9 @@ def test_cached_forward_matches_torch_and_bruteforce(shape):
         step_logits.append(o.last_logits)
     ref_t = torch_forward(shape, w, seq[:-1])
     ref_b = o.full_recompute_logits(seq[:-1])
-    tol = 1e-9 if shape.dtype == "f32" else 0.15       # bf16 K/V: a flipped rounding moves a logit by ~1e-2
+    # the references round K/V to bf16 at the same point (after the rotation), so fp64 summation order is the only
+    # difference; a forgotten rounding, or one applied before the rotation, moves logits by ~1e-2 and fails here
+    tol = 1e-9
     for i, z in enumerate(step_logits):
         row = len(prompt) - 1 + i
         assert np.max(np.abs(z - ref_t[row])) < tol, (i, np.max(np.abs(z - ref_t[row])))
@@ -214,3 +216,60 @@ def test_workload_calibration_recorded_range():
     ks = [r["k"] for r in o.log]
     assert any(r["k"] < r["n_drafted"] for r in o.log) and any(r["k"] == r["n_drafted"] for r in o.log)
     assert 1.2 < ko.compression_rate(o.S) < 4.0
+
+
+# ---------------------------------------------------------------- where K and V are rounded for bf16 models
+
+def _bf16_by_hand(x: float) -> float:
+    """Nearest-even rounding of a Python float to bfloat16, on the bits of its fp32 value."""
+    import struct
+    bits = struct.unpack("<I", struct.pack("<f", x))[0]
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return struct.unpack("<f", struct.pack("<I", bits))[0]
+
+
+def test_kv_cache_stores_bf16_of_rotated_k_and_of_v():
+    """bf16 models keep K and V in bf16: K is rotated first and rounded when stored, V is rounded when stored, and
+    nothing else is rounded.  Two heads of four dimensions, position 3, every value worked out with scalar
+    arithmetic; the inputs are chosen so that leaving the rounding out, or rounding K before the rotation, gives
+    different stored values."""
+    import math
+    H, hd, d, pos, theta = 2, 4, 8, 3, 10000.0
+    shape = MICRO_BF.with_(d_model=d, n_heads=H, head_dim=hd, max_seq=8, rope_theta=theta)
+    o = ko.KangarooOracle.__new__(ko.KangarooOracle)
+    o.s, o.dt, o.d, o.H, o.hd = shape, np.dtype(np.float64), d, H, hd
+    cache = ko.KVCache(8, H, hd, np.float64, True)
+    cache.length = pos                                    # rows 0..2 stay zero: they only add exp(0) terms below
+    q = [0.3, -1.1, 0.7, 0.2, -0.4, 0.9, 1.3, -0.6]
+    k = [1.2345678, -0.7654321, 2.3456789, 0.1234567, -1.1111111, 0.3333333, 0.9876543, -2.2222222]
+    v = [0.1111111, 1.7777777, -0.5555555, 3.1415926, -2.7182818, 0.5772156, 1.4142135, -1.7320508]
+    qkv = np.array([q + k + v], np.float64)
+    out = o.attention_core(qkv, pos, cache)
+    assert cache.length == pos + 1
+
+    def rot(x, h):                                        # pairs (i, i + hd/2), angle pos * theta^(-2i/hd)
+        r = [0.0] * hd
+        for i in range(hd // 2):
+            a = pos * theta ** (-2.0 * i / hd)
+            x1, x2 = x[h * hd + i], x[h * hd + i + hd // 2]
+            r[i] = x1 * math.cos(a) - x2 * math.sin(a)
+            r[i + hd // 2] = x2 * math.cos(a) + x1 * math.sin(a)
+        return r
+
+    k_rot = [rot(k, h) for h in range(H)]
+    k_exp = [[_bf16_by_hand(x) for x in k_rot[h]] for h in range(H)]
+    v_exp = [[_bf16_by_hand(v[h * hd + e]) for e in range(hd)] for h in range(H)]
+    assert np.array_equal(cache.k[pos], np.array(k_exp)) and np.array_equal(cache.v[pos], np.array(v_exp))
+    # the two plausible mistakes give other values on this input
+    k_unrounded = np.array(k_rot)
+    k_round_first = np.array([rot([_bf16_by_hand(x) for x in k], h) for h in range(H)])
+    assert not np.array_equal(cache.k[pos], k_unrounded) and np.max(np.abs(cache.k[pos] - k_unrounded)) > 1e-4
+    assert np.max(np.abs(cache.k[pos] - k_round_first)) > 1e-4
+    assert np.max(np.abs(cache.v[pos] - np.array(v).reshape(H, hd))) > 1e-4
+    # and the attention output uses the stored (rounded) row: softmax over three zero keys and the new key
+    for h in range(H):
+        qr = rot(q, h)
+        s_new = sum(a * b for a, b in zip(qr, k_exp[h])) / math.sqrt(hd)
+        w_new = math.exp(s_new) / (3.0 + math.exp(s_new))
+        for e in range(hd):
+            assert abs(out[0, h * hd + e] - w_new * v_exp[h][e]) < 1e-12
