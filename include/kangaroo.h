@@ -34,7 +34,7 @@ typedef enum {
     KG_E_NOMEM = -3,     /* arena too small */
     KG_E_SEQ_FULL = -4,  /* the sequence would exceed max_seq */
     KG_E_CUDA = -5,      /* a CUDA runtime call failed */
-    KG_E_TIMEOUT = -6,   /* a bounded device-side wait expired; the model must be re-initialised */
+    KG_E_TIMEOUT = -6,   /* a bounded device-side wait expired; the model must be re-initialised (kg_init_model) */
     KG_E_LIMIT = -7      /* a size exceeds what a fixed-capacity entry point (kg_op_lm_head_noalloc) can hold */
 } kg_status;
 
@@ -57,8 +57,8 @@ typedef struct {
     float init_std, embed_std, deep_resid_scale, adapter_resid_scale, gain_std;
 } kg_config;
 
-/* Borrowed device pointers to caller-provided weights (optional).  Arrays are HOST arrays of
- * device pointers.  Index L (= n_layers) of wqkv / wo / g1 / g2 is the adapter (g1 = input norm
+/* Borrowed device pointers to caller-provided weights (optional), each 16-byte aligned (else KG_E_ARG:
+ * the kernels read them with 16-byte bulk copies).  Arrays are HOST arrays of device pointers.  Index L (= n_layers) of wqkv / wo / g1 / g2 is the adapter (g1 = input norm
  * gain, g2 = last norm gain).  Matrices have the model's storage dtype, gains are fp32. */
 typedef struct {
     const void* embed_dev;                   /* [V, d] */
@@ -116,9 +116,10 @@ int kg_reset(kg_model* m);
 
 /* All L layers over the prompt, the adapter's K/V for every prompt position, and
  * x_0 = argmax M^b(. | prompt) (Figure 2's starting point).  Requires a reset model.
- * kg_prefill copies the prompt from the host; if first_token_host != NULL it synchronises the
- * stream and returns x_0.  kg_prefill_device reads prompt ids already in device memory and
- * never synchronises. */
+ * kg_prefill copies the prompt from the host (ids outside [0, vocab) -> KG_E_ARG, nothing launched); if
+ * first_token_host != NULL it synchronises the stream and returns x_0.  kg_prefill_device reads prompt ids
+ * already in device memory and never synchronises: an id outside [0, vocab) is caught on the device (the
+ * embedding lookup stays in bounds) and the next call that synchronises returns KG_E_ARG; kg_reset clears it. */
 int kg_prefill(kg_model* m, const int32_t* prompt_host, int32_t n, int32_t* first_token_host);
 int kg_prefill_device(kg_model* m, const int32_t* prompt_dev, int32_t n);
 
@@ -170,9 +171,22 @@ int kg_read_weight(kg_model* m, const char* name, int32_t layer, uint64_t offset
  * x_0 = token, and, if n_d >= 0, a pending draft of n_d seeded tokens with N(0,1) early features. */
 int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t seed);
 
+/* ---- test hooks (no part of the method; used by the parity and failure-path tests) ----------------
+ * kg_debug_force_simple: route a bf16 model's linear operators through the plain (non tensor-core) path, a
+ *   cross-check of the streamed path.  kg_debug_force_simple_ops: the same for the single-operator calls.
+ * kg_debug_set_wait_budget: every wait inside a kernel (grid barrier, weight ring) gives up after this many
+ *   milliseconds (default about 3 s) and the launch ends with KG_E_TIMEOUT in the state word.
+ * kg_debug_skip_barrier_arrival: in the NEXT launch, CTA `cta` leaves out its first grid-barrier arrival, so that
+ *   every CTA's wait runs into the budget: the host-injected way to exercise the time-out path.  Nothing traps or
+ *   faults; all CTAs return, the stream stays usable, and the model answers KG_E_TIMEOUT until it is re-initialised. */
+int kg_debug_force_simple(kg_model* m, int on);
+int kg_debug_force_simple_ops(int on);
+int kg_debug_set_wait_budget(kg_model* m, double milliseconds);
+int kg_debug_skip_barrier_arrival(kg_model* m, int cta);
+
 /* ---- single operators on caller buffers (unit tests and microbenchmarks) ------------------------
- * All pointers are device pointers; `scratch_dev` must hold kg_op_scratch_bytes() bytes; the
- * call is asynchronous on `cuda_stream`.  dtype is KG_F32 or KG_BF16 and is the type of W / KV. */
+ * All pointers are device pointers, 16-byte aligned (int32 arrays: 4-byte), else KG_E_ARG; `scratch_dev` must hold
+ * kg_op_scratch_bytes() bytes; the call is asynchronous on `cuda_stream`.  dtype is KG_F32 or KG_BF16 and is the type of W / KV. */
 size_t kg_op_scratch_bytes(void);
 
 /* out[M, N] = (resid ? resid : 0) + RMSNorm(x; gain, eps) W^T   (gain == NULL: no norm)
@@ -193,7 +207,7 @@ int kg_op_lm_head(int32_t dtype, const void* W_head_dev, int32_t V, int32_t K, c
  * a deployment convenience).  It is for callers that cannot obtain device memory at the time of the call -
  * code running while a memory pool is frozen or exhausted, inside a plugin whose host forbids cudaMalloc, or
  * in an error path that must still produce a token.  The per-CTA partial results that kg_op_lm_head keeps in
- * `scratch_dev` (per-CTA partial results, and the repacked copy of the input rows) lives here in a 592 KB array
+ * `scratch_dev` (per-CTA partial results, and the repacked copy of the input rows) live here in a 592 KB array
  * that is part of the library image, so every GPU that loads the library holds those 592 KB until the process exits.
  * Limits: M <= KG_M_MAX rows, K <= 8192 and a device with at most 256 SMs; anything larger returns KG_E_LIMIT.
  * V is not limited: W, x and the outputs remain caller memory.

@@ -24,6 +24,7 @@ EXPORTS = [
     "kg_draft", "kg_verify", "kg_decode", "kg_decode_ar", "kg_generate", "kg_read_tokens", "kg_read_S", "kg_read_round_log",
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
     "kg_op_lm_head", "kg_op_lm_head_noalloc", "kg_op_attention", "kg_strerror",
+    "kg_debug_force_simple", "kg_debug_force_simple_ops", "kg_debug_set_wait_budget", "kg_debug_skip_barrier_arrival",
 ]
 
 
@@ -114,6 +115,8 @@ def load():
     lib.kg_strerror.argtypes = [C.c_int]
     lib.kg_debug_force_simple.argtypes = [vp, C.c_int]
     lib.kg_debug_force_simple_ops.argtypes = [C.c_int]
+    lib.kg_debug_set_wait_budget.argtypes = [vp, C.c_double]
+    lib.kg_debug_skip_barrier_arrival.argtypes = [vp, C.c_int]
     _lib = lib
     return lib
 
@@ -146,7 +149,11 @@ def config_from_shape(shape, debug_logits=False, page_shuffle=False) -> KgConfig
 class KangarooModel:
     """A model living in a torch-owned device arena, driven through the C ABI."""
 
-    def __init__(self, shape, debug_logits=False, page_shuffle=False, device="cuda:0", stream=None):
+    def __init__(self, shape, debug_logits=False, page_shuffle=False, device="cuda:0", stream=None, weights=None,
+                 arena=None):
+        """weights: None (the library fills seeded synthetic weights into the arena) or the nested dict of host
+        arrays the input generator makes; those are uploaded as torch tensors and handed over as borrowed
+        pointers (kg_weights).  arena: an existing uint8 device tensor to build the model in."""
         import torch
         self.torch = torch
         self.lib = load()
@@ -154,16 +161,54 @@ class KangarooModel:
         self.cfg = config_from_shape(shape, debug_logits, page_shuffle)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
-        nbytes = self.lib.kg_workspace_bytes(C.byref(self.cfg), 1)
+        nbytes = self.lib.kg_workspace_bytes(C.byref(self.cfg), 0 if weights is not None else 1)
         if nbytes == 0:
             raise KgError(KG_E_ARG, "kg_workspace_bytes")
-        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        if arena is not None and arena.numel() < nbytes:
+            raise KgError(KG_E_NOMEM, "arena")
+        self.arena = arena if arena is not None else torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        kw = self._borrowed(weights) if weights is not None else None
         h = C.c_void_p()
-        _check(self.lib.kg_init_model(C.byref(self.cfg), None, self.arena.data_ptr(), nbytes,
-                                      self.stream.cuda_stream, C.byref(h)), "kg_init_model")
+        _check(self.lib.kg_init_model(C.byref(self.cfg), C.byref(kw) if kw is not None else None, self.arena.data_ptr(),
+                                      self.arena.numel(), self.stream.cuda_stream, C.byref(h)), "kg_init_model")
         self.h = h
         self.arena_bytes = nbytes
+
+    def _borrowed(self, w):
+        """Uploads the host weights and returns the kg_weights table of device pointers (tensors kept alive here)."""
+        torch = self.torch
+        mdt = torch.bfloat16 if self.shape.dtype == "bf16" else torch.float32
+        self._wt = []
+
+        def up(a, dt):
+            t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(self.device).to(dt).contiguous()
+            self._wt.append(t)
+            return t.data_ptr()
+
+        L = self.shape.n_layers
+        blocks = list(w["layers"]) + [w["adapter"]]
+        kw = KgWeights()
+        kw.embed_dev, kw.head_dev = up(w["embed"], mdt), up(w["head"], mdt)
+        kw.g_final_dev = up(w["g_final"], torch.float32)
+
+        def table(name, dt, adapter_name=None, with_adapter=True):
+            arr = (C.c_void_p * (L + 1))()
+            for i, blk in enumerate(blocks):
+                if i == L and not with_adapter:
+                    arr[i] = None
+                else:
+                    arr[i] = up(blk[adapter_name if (i == L and adapter_name) else name], dt)
+            self._wt.append(arr)
+            return arr
+
+        kw.wqkv_dev, kw.wo_dev = table("wqkv", mdt), table("wo", mdt)
+        kw.wgate_dev = table("wgate", mdt, with_adapter=False)
+        kw.wup_dev = table("wup", mdt, with_adapter=False)
+        kw.wdown_dev = table("wdown", mdt, with_adapter=False)
+        kw.g1_dev = table("g1", torch.float32, adapter_name="g_in")
+        kw.g2_dev = table("g2", torch.float32, adapter_name="g_last")
+        return kw
 
     def close(self):
         if self.h:
@@ -274,6 +319,12 @@ class KangarooModel:
 
     def force_simple(self, on):
         _check(self.lib.kg_debug_force_simple(self.h, int(on)), "kg_debug_force_simple")
+
+    def set_wait_budget(self, milliseconds):
+        _check(self.lib.kg_debug_set_wait_budget(self.h, float(milliseconds)), "kg_debug_set_wait_budget")
+
+    def skip_barrier_arrival(self, cta):
+        _check(self.lib.kg_debug_skip_barrier_arrival(self.h, int(cta)), "kg_debug_skip_barrier_arrival")
 
 
 # ---- single operators ---------------------------------------------------------------------------

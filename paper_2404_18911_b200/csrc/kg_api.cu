@@ -190,14 +190,27 @@ Layout make_layout(const kg_config* c, int own_weights, int nctas) {
     return L;
 }
 
-int g_sm_count = 0;
+// SM count of the current device (one CTA per SM in every launch), looked up once per device.
+constexpr int MAX_DEVICES = 64;
+int g_sm_count[MAX_DEVICES] = {0};
 int sm_count() {
-    if (g_sm_count > 0) return g_sm_count;
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev >= 0 && dev < MAX_DEVICES && g_sm_count[dev] > 0) return g_sm_count[dev];
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
-    g_sm_count = n;
+    if (dev >= 0 && dev < MAX_DEVICES) g_sm_count[dev] = n;
     return n;
+}
+
+// Device pointers handed in by the caller feed 16-byte bulk copies and vector loads: anything less aligned would
+// fault on the device, so it is refused on the host.
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Token ids that arrive in device memory cannot be checked on the host: one thread per id records an argument
+// error in the state word (the embedding lookup itself keeps every access in bounds).
+__global__ void check_tokens_kernel(const int* toks, int n, int vocab, State* st) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n && (unsigned)toks[i] >= (unsigned)vocab) atomicCAS(&st->status, 0, (int)KG_E_ARG);
 }
 
 }  // namespace
@@ -212,6 +225,9 @@ struct kg_model {
     size_t smem;
     bool own_weights;
     bool prefilled, pending, ar_used, dead;
+    unsigned long long wait_clk;   // budget of a device-side wait, in SM clocks
+    int skip_arrival;              // test hook, consumed by the next launch
+    cudaEvent_t ev0, ev1;          // timing of the decode loop in kg_generate, created on first use
     int gamma_pending;
     long long P_upper;      // upper bound of the device-side position P
     int force_simple;
@@ -244,6 +260,9 @@ static int launch_program(kg_model* m, const Program& pg) {
     CK(cudaMemsetAsync(m->dev.bar, 0, BAR_BYTES, m->stream));
     Program p = pg;
     p.force_simple = m->force_simple;
+    p.wait_clk = m->wait_clk;
+    p.skip_arrival = m->skip_arrival;
+    m->skip_arrival = 0;
     void* args[] = {(void*)&m->dev, (void*)&p};
     CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(BLOCK_THREADS), args, m->smem, m->stream));
     return KG_OK;
@@ -255,7 +274,13 @@ static int launch(kg_model* m, const Program& pg) {
 static int read_state(kg_model* m, State* out) {
     CK(cudaMemcpyAsync(out, m->dev.st, sizeof(State), cudaMemcpyDeviceToHost, m->stream));
     CK(cudaStreamSynchronize(m->stream));
-    if (out->status != 0) { m->dead = true; return out->status; }
+    if (out->status == ST_TIMEOUT) { m->dead = true; return KG_E_TIMEOUT; }
+    if (out->status != 0) {
+        // an argument error found on the device (a token id outside the vocabulary): the sequence is unusable until
+        // kg_reset, which also clears the state word; the weights are untouched
+        m->prefilled = m->pending = false; m->ar_used = true;
+        return out->status;
+    }
     return KG_OK;
 }
 
@@ -301,6 +326,14 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     if (w) {
         if (!w->embed_dev || !w->head_dev || !w->g_final_dev || !w->wqkv_dev || !w->wo_dev || !w->wgate_dev ||
             !w->wup_dev || !w->wdown_dev || !w->g1_dev || !w->g2_dev) return KG_E_ARG;
+        if (!aligned16(w->embed_dev) || !aligned16(w->head_dev) || !aligned16(w->g_final_dev)) return KG_E_ARG;
+        for (int i = 0; i <= cfg->n_layers; ++i) {
+            const bool layer = i < cfg->n_layers;
+            if (!w->wqkv_dev[i] || !w->wo_dev[i] || !w->g1_dev[i] || !w->g2_dev[i] ||
+                (layer && (!w->wgate_dev[i] || !w->wup_dev[i] || !w->wdown_dev[i]))) return KG_E_ARG;
+            if (!aligned16(w->wqkv_dev[i]) || !aligned16(w->wo_dev[i]) || !aligned16(w->g1_dev[i]) || !aligned16(w->g2_dev[i]) ||
+                (layer && (!aligned16(w->wgate_dev[i]) || !aligned16(w->wup_dev[i]) || !aligned16(w->wdown_dev[i])))) return KG_E_ARG;
+        }
     }
     const int nctas = sm_count();
     const int own = w ? 0 : 1;
@@ -313,6 +346,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     m->cfg = *cfg; m->lay = lay; m->arena = base; m->stream = (cudaStream_t)cuda_stream; m->nctas = nctas;
     m->own_weights = own != 0; m->prefilled = m->pending = m->ar_used = m->dead = false;
     m->gamma_pending = 0; m->P_upper = 0; m->force_simple = 0;
+    m->wait_clk = WAIT_TIMEOUT_CLK; m->skip_arrival = 0; m->ev0 = m->ev1 = nullptr;
     m->smem = SMEM_TOTAL;
 
     const bool bf = cfg->dtype == KG_BF16;
@@ -332,7 +366,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     for (int i = 0; i < cfg->head_dim / 2; ++i)
         D.inv_freq[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
     auto P = [&](size_t off) { return base + off; };
-    D.st = (State*)P(lay.off_st); D.bar = (unsigned*)P(lay.off_bar);
+    D.st = (State*)P(lay.off_st); D.bar = (unsigned long long*)P(lay.off_bar);
     D.layers = (const LayerW*)P(lay.off_layers); D.page_table = (const int*)P(lay.off_pt);
     D.kcache = P(lay.off_kc); D.vcache = P(lay.off_vc);
     D.h = (float*)P(lay.off_h); D.feat = (float*)P(lay.off_feat); D.abuf = (float*)P(lay.off_abuf);
@@ -372,7 +406,6 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
             lw.wup = i < nl ? w->wup_dev[i] : nullptr;
             lw.wdown = i < nl ? w->wdown_dev[i] : nullptr;
             lw.g1 = w->g1_dev[i]; lw.g2 = w->g2_dev[i];
-            if (!lw.wqkv || !lw.wo || !lw.g1 || !lw.g2 || (i < nl && (!lw.wgate || !lw.wup || !lw.wdown))) { delete m; return KG_E_ARG; }
         }
     }
     cudaStream_t s = m->stream;
@@ -401,6 +434,8 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
 
 extern "C" int kg_free_model(kg_model* m) {
     if (!m) return KG_E_ARG;
+    if (m->ev0) cudaEventDestroy(m->ev0);
+    if (m->ev1) cudaEventDestroy(m->ev1);
     delete m;
     return KG_OK;
 }
@@ -449,7 +484,10 @@ extern "C" int kg_prefill_device(kg_model* m, const int32_t* prompt_dev, int32_t
     if (m->dead) return KG_E_TIMEOUT;
     if (m->prefilled || m->ar_used) return KG_E_STATE;
     if (n + 1 > m->cfg.max_seq) return KG_E_SEQ_FULL;
+    if (reinterpret_cast<uintptr_t>(prompt_dev) & 3u) return KG_E_ARG;
     CK(cudaMemcpyAsync((void*)m->dev.prompt, prompt_dev, sizeof(int32_t) * n, cudaMemcpyDeviceToDevice, m->stream));
+    check_tokens_kernel<<<(n + 255) / 256, 256, 0, m->stream>>>(m->dev.prompt, n, m->cfg.vocab, m->dev.st);
+    CK(cudaGetLastError());
     return prefill_common(m, n);
 }
 
@@ -622,11 +660,13 @@ extern "C" int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_pr
     CK(cudaMemcpyAsync((void*)m->dev.prompt, prompt_host, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->stream));
     r = prefill_common(m, n_prompt);
     if (r != KG_OK) return r;
-    cudaEvent_t e0 = nullptr, e1 = nullptr;
     const bool timed = stats != nullptr;
-    if (timed) { CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1)); CK(cudaEventRecord(e0, m->stream)); }
+    if (timed) {
+        if (!m->ev0) { CK(cudaEventCreate(&m->ev0)); CK(cudaEventCreate(&m->ev1)); }      // once per model
+        CK(cudaEventRecord(m->ev0, m->stream));
+    }
     r = kg_decode(m, max_new, eta, gamma, stop_mode, nullptr);
-    if (timed && r == KG_OK) cudaEventRecord(e1, m->stream);
+    if (timed && r == KG_OK) cudaEventRecord(m->ev1, m->stream);
     State st;
     if (r == KG_OK) r = read_state(m, &st);
     if (r == KG_OK) {
@@ -642,12 +682,10 @@ extern "C" int kg_generate(kg_model* m, const int32_t* prompt_host, int32_t n_pr
             if (r == KG_OK) {
                 fill_stats(m, st, S, max_new, stats);
                 float ms = 0.f;
-                if (cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess) stats->ms_decode = ms;
+                if (cudaEventElapsedTime(&ms, m->ev0, m->ev1) == cudaSuccess) stats->ms_decode = ms;
             }
         }
     }
-    if (e0) cudaEventDestroy(e0);
-    if (e1) cudaEventDestroy(e1);
     return r;
 }
 
@@ -731,10 +769,25 @@ extern "C" int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t
     return KG_OK;
 }
 
-// Test hook (not in the public header): route bf16 linears through the plain path.
 extern "C" int kg_debug_force_simple(kg_model* m, int on) {
     if (!m) return KG_E_ARG;
     m->force_simple = on ? 1 : 0;
+    return KG_OK;
+}
+
+extern "C" int kg_debug_set_wait_budget(kg_model* m, double milliseconds) {
+    if (!m || !(milliseconds > 0.0) || milliseconds > 60000.0) return KG_E_ARG;
+    int dev = 0, khz = 0;
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+    m->wait_clk = (unsigned long long)(milliseconds * (double)khz);      // kHz = clocks per millisecond
+    if (m->wait_clk < 1000ull) m->wait_clk = 1000ull;
+    return KG_OK;
+}
+
+extern "C" int kg_debug_skip_barrier_arrival(kg_model* m, int cta) {
+    if (!m || cta < 0 || cta >= m->nctas) return KG_E_ARG;
+    m->skip_arrival = cta + 1;
     return KG_OK;
 }
 
@@ -821,6 +874,8 @@ extern "C" int kg_op_linear(int32_t dtype, const void* W, const void* W2, int32_
                             const float* resid, int32_t swiglu, float* out, void* scratch, void* stream) {
     if (!W || !x || !out || !scratch) return KG_E_ARG;
     if (swiglu && !W2) return KG_E_ARG;
+    if (!aligned16(W) || !aligned16(W2) || !aligned16(x) || !aligned16(gain) || !aligned16(resid) || !aligned16(out) ||
+        !aligned16(scratch)) return KG_E_ARG;
     LinArgs a{};
     a.W = W; a.W2 = swiglu ? W2 : nullptr; a.N = N; a.K = K; a.x = x; a.ldx = K; a.M = M; a.gain = gain; a.eps = eps;
     a.resid = resid; a.ldr = N; a.out = out; a.ldo = N;
@@ -833,6 +888,8 @@ extern "C" int kg_op_lm_head(int32_t dtype, const void* W, int32_t V, int32_t K,
                              const float* gain, float eps, float logit_scale,
                              int32_t* tok, float* p, float* logits, void* scratch, void* stream) {
     if (!W || !x || !tok || !p || !scratch) return KG_E_ARG;
+    if (!aligned16(W) || !aligned16(x) || !aligned16(gain) || !aligned16(logits) || !aligned16(scratch) ||
+        (reinterpret_cast<uintptr_t>(tok) & 3u) || (reinterpret_cast<uintptr_t>(p) & 3u)) return KG_E_ARG;
     if (sm_count() > 1024) return KG_E_ARG;
     OpScratch sc = op_layout();
     LinArgs a{};
@@ -857,6 +914,7 @@ constexpr size_t NOALLOC_OFF_XPK = sizeof(float4) * NOALLOC_MAX_CTAS * KG_M_MAX;
 constexpr size_t NOALLOC_OFF_SSQ = NOALLOC_OFF_XPK + 4 * (size_t)KG_M_MAX * NOALLOC_MAX_K;        // packed input rows: 512 KB
 constexpr size_t NOALLOC_BYTES = NOALLOC_OFF_SSQ + 4 * (size_t)KG_M_MAX * NOALLOC_MAX_CTAS;       // sums of squares: 16 KB
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+static_assert(NOALLOC_MAX_DEVICES <= MAX_DEVICES, "per-device tables");
 void* g_noalloc_addr[NOALLOC_MAX_DEVICES] = {nullptr};
 
 // Device address of the static scratch on the current device.  In host code the array's name is only a
@@ -879,6 +937,8 @@ extern "C" int kg_op_lm_head_noalloc(int32_t dtype, const void* W, int32_t V, in
                                      const float* gain, float eps, float logit_scale,
                                      int32_t* tok, float* p, float* logits, void* stream) {
     if (!W || !x || !tok || !p) return KG_E_ARG;
+    if (!aligned16(W) || !aligned16(x) || !aligned16(gain) || !aligned16(logits) ||
+        (reinterpret_cast<uintptr_t>(tok) & 3u) || (reinterpret_cast<uintptr_t>(p) & 3u)) return KG_E_ARG;
     if (M > KG_M_MAX || K > NOALLOC_MAX_K || sm_count() > NOALLOC_MAX_CTAS) return KG_E_LIMIT;
     void* scratch = nullptr;
     int r = noalloc_scratch(&scratch);
@@ -901,6 +961,8 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
                                float* out, void* scratch, void* stream) {
     if (!qkv || !kc || !vc || !page_table || !out || !scratch) return KG_E_ARG;
     if (dtype != KG_F32 && dtype != KG_BF16) return KG_E_ARG;
+    if (!aligned16(qkv) || !aligned16(kc) || !aligned16(vc) || !aligned16(out) || !aligned16(scratch) ||
+        (reinterpret_cast<uintptr_t>(page_table) & 3u)) return KG_E_ARG;
     if (M < 1 || M > KG_M_MAX || pos0 < 0 || H < 1 || H > 256 || (hd != 32 && hd != 64 && hd != 128) || page_size < 1 ||
         (page_size & (page_size - 1))) return KG_E_ARG;
     if ((size_t)H * hd > 8192) return KG_E_ARG;

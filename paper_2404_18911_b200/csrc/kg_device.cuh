@@ -19,14 +19,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-// Timeline hook for profiling builds (a translation unit may define it before including this file).
-#ifndef KG_PROBE
-#define KG_PROBE(tag) do { } while (0)
-#endif
-#ifndef KG_PROBE_INIT
-#define KG_PROBE_INIT() do { } while (0)
-#endif
-
 namespace kg {
 
 constexpr int M_MAX = 16;          // rows per pass
@@ -55,7 +47,7 @@ constexpr int SIMPLE_XS_BYTES = SMEM_TOTAL - RING_OFF - 4096;
 
 constexpr int BAR_RELEASE = 32;                          // word index of the grid barrier's release word (its own 128-byte line)
 constexpr int BAR_BYTES = 256;
-constexpr unsigned long long WAIT_TIMEOUT_CLK = 6000000000ull;   // ~3 s at 1.9 GHz
+constexpr unsigned long long WAIT_TIMEOUT_CLK = 6000000000ull;   // default budget of a device-side wait: ~3 s at 1.9 GHz
 
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_HEAD = 3 };
 enum { ST_OK = 0, ST_TIMEOUT = -6 };
@@ -124,7 +116,7 @@ struct Dev {
     int* out_tokens; int* S; int* round_log;   // [max_seq], [max_seq], [max_seq][4]
     const int* prompt;             // device copy of the prompt
     State* st;
-    unsigned* bar;                 // grid barrier arrival counter (zeroed before every launch)
+    unsigned long long* bar;       // grid barrier arrival counter (zeroed before every launch)
     double inv_freq[HD_MAX / 2];   // theta^(-2i/hd)
 };
 
@@ -154,8 +146,10 @@ static_assert(sizeof(Ctrl) <= CTRL_BYTES - 16, "control block too large");
 // role's barriers; reading it never touches the per-thread stack.
 struct Ctx {
     int cta, nctas;
-    unsigned bar_target;           // arrivals expected at the next grid barrier (thread 0 only)
-    State* st; unsigned* bar;
+    unsigned long long bar_target; // arrivals expected at the next grid barrier (thread 0 only)
+    unsigned long long wait_clk;   // clocks after which a wait of this launch gives up
+    State* st; unsigned long long* bar;
+    int skip_arrival;              // test hook: 1 + index of the CTA that leaves out its first grid-barrier arrival (0: none)
     char* smem;
     Ctrl* ctl;
     bool grid;                     // false: single-operator test kernel, grid barriers are CTA barriers
@@ -169,9 +163,9 @@ struct Ctx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
@@ -204,7 +198,7 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsign
 
 // The top bit of the grid barrier's arrival counter tells every CTA that some wait has given up: they learn it from
 // the word they poll anyway, without a second load.
-constexpr unsigned BAR_ABORT = 0x80000000u;
+constexpr unsigned long long BAR_ABORT = 0x8000000000000000ull;
 __device__ __forceinline__ void record_timeout(Ctx& c, int where) {
     *(volatile int*)&c.ctl->abort = 1;
     if (c.st) {
@@ -224,7 +218,7 @@ __device__ __forceinline__ bool mbar_wait(Ctx& c, unsigned long long* bar, unsig
         if (c.producer) __nanosleep(200);
         if (((++spins) & 63u) == 0u) {
             if (*(volatile int*)&c.ctl->abort) return false;
-            if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); return false; }
+            if ((unsigned long long)(clock64() - t0) > c.wait_clk) { record_timeout(c, where); return false; }
         }
     }
     return true;
@@ -273,18 +267,19 @@ __device__ __forceinline__ bool arg_better(float za, int ia, float zb, int ib) {
 
 // ------------------------------------------------------------------------------------ CTA set-up
 // Called by every thread of the CTA at kernel start; returns the context of the thread's role.
-__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, bool grid) {
+__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned long long* bar, bool grid,
+                                         unsigned long long wait_clk = WAIT_TIMEOUT_CLK, int skip_arrival = 0) {
     static_assert(sizeof(Ctx) <= 128, "context slot too small");
     Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
     const bool producer = threadIdx.x >= NTHREADS;
     Ctx& c = *reinterpret_cast<Ctx*>(producer ? ctl->ctx_prod : ctl->ctx_cons);
     if (threadIdx.x == 0 || threadIdx.x == NTHREADS) {
         c.cta = blockIdx.x; c.nctas = gridDim.x; c.bar_target = 0; c.st = st; c.bar = bar; c.smem = smem;
+        c.wait_clk = wait_clk; c.skip_arrival = skip_arrival;
         c.ctl = ctl; c.grid = grid;
         c.producer = producer;
         c.slot = 0; c.phase = 0; c.issued = 0; c.mail_phase = 0;
     }
-    KG_PROBE_INIT();
     if (threadIdx.x == 0) {
         for (int i = 0; i < RING; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], NWARPS); }
         mbar_init(&ctl->mail, 1);
@@ -302,23 +297,23 @@ __device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, b
 __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
     if (!c.grid) { cta_sync(); return *(volatile int*)&c.ctl->abort == 0; }
     cta_sync();
-    KG_PROBE(1);
     if (threadIdx.x == 0) {
-        // bar[0] counts arrivals (monotonic over the launch, far below 2^31): one release-add, then poll until every CTA
-        // has arrived or the abort bit appears
-        c.bar_target += (unsigned)c.nctas;
-        const unsigned gen = c.bar_target;
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.bar) : "memory");
+        // bar[0] counts arrivals (64 bits, monotonic over the launch): one release-add, then poll until every CTA has
+        // arrived or the abort bit appears
+        c.bar_target += (unsigned long long)c.nctas;
+        const unsigned long long gen = c.bar_target;
+        if (c.skip_arrival == c.cta + 1) c.skip_arrival = 0;        // test hook: this arrival never happens
+        else asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(c.bar) : "memory");
         int ok = 1;
         {
             const long long t0 = clock64();
             unsigned spins = 0;
             while (true) {
-                const unsigned v = ld_acquire_u32(c.bar);
+                const unsigned long long v = ld_acquire_u64(c.bar);
                 if (v & BAR_ABORT) { ok = 0; break; }
-                if ((int)(v - gen) >= 0) break;
+                if (v >= gen) break;
                 if (((++spins) & 63u) == 0u) {
-                    if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) { record_timeout(c, where); ok = 0; break; }
+                    if ((unsigned long long)(clock64() - t0) > c.wait_clk) { record_timeout(c, where); ok = 0; break; }
                 }
             }
         }
@@ -326,7 +321,6 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
         c.ctl->sync_ok = ok;
     }
     cta_sync();
-    KG_PROBE(2);
     return *(volatile int*)&c.ctl->sync_ok != 0;
 }
 
@@ -466,7 +460,6 @@ __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
                 if (lane == 0) mbar_arrive_expect_tx(&ctl->full[slot], (unsigned)(nvalid * len * 2));
                 __syncwarp();
                 if (lane < nvalid) bulk_g2s(ring + (size_t)slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &ctl->full[slot]);
-                KG_PROBE(30);
                 issued++;
                 if (++slot == RING) { slot = 0; phase ^= 1u; }
             }
@@ -485,7 +478,7 @@ __device__ void ring_drain(Ctx& c) {
         if (--s < 0) { s = RING - 1; ph ^= 1u; }
         const long long t0 = clock64();
         while (!mbar_try_wait(&c.ctl->full[s], ph)) {
-            if ((unsigned long long)(clock64() - t0) > WAIT_TIMEOUT_CLK) break;
+            if ((unsigned long long)(clock64() - t0) > c.wait_clk) break;
         }
     }
 }
@@ -589,7 +582,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
     bool ok = true;
     int buf = 0;
     float ssq_acc = 0.f;
-    KG_PROBE(10);
 
     // ---- fetched early, used in the epilogue: the input rows' sums of squares, residual values, output gains.
     // The requests go out right behind the first phase's fragment loads, which the first MMA waits for.
@@ -662,7 +654,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                     }
                 }
             }
-            KG_PROBE(11);
             // ---- the row groups of this phase, two stages (16 weight rows) at a time
             const uint32_t a_lane = (uint32_t)((lane & 7) * ST_ROW_BYTES + (warp * NS * 16 + (lane >> 4) * 8) * 2);
             for (int si = 0; si < nst; si += 2) {
@@ -675,7 +666,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                 for (int q = 0; q < 4; ++q) { acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f; }
                 if (ok) ok = mbar_wait(c, &ctl->full[slot_a], phase, 41);
                 if (ok && two) ok = mbar_wait(c, &ctl->full[slot_b], phase_b, 41);
-                KG_PROBE(12);
                 if (ok) {
                     // ldmatrix x4: matrices 0, 2 = rows 0-7 (first stage), 1, 3 = rows 8-15 (second stage); k halves 0-7 | 8-15
                     const uint32_t a_base = smem_u32(ring + (size_t)((lane & 8) ? slot_b : slot_a) * SLOT_BYTES) + a_lane;
@@ -699,7 +689,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                     }
                 }
                 __syncwarp();
-                KG_PROBE(13);
                 if (ok && lane == 0) { mbar_arrive(&ctl->empty[slot_a]); if (two) mbar_arrive(&ctl->empty[slot_b]); }
                 slot = slot_b; phase = phase_b;
                 if (++slot == RING) { slot = 0; phase ^= 1u; }
@@ -748,7 +737,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                         }
                     }
                 }
-                KG_PROBE(14);
                 buf ^= 1;
             }
         }
@@ -795,7 +783,6 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
             emit_rows(a, wk, sc0, nu, prefetched && sc0 == pl.u0, ssq_acc);
         }
         cta_sync();                                  // acc_s is rewritten by the next superchunk / operator
-        KG_PROBE(15);
     }
     if (a.epi == EPI_HEAD && lane == 0) {
 #pragma unroll
@@ -1081,7 +1068,6 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) { AttLoad<WT, DPL>::cvt(kr[j], kv[j]); AttLoad<WT, DPL>::cvt(vr[j], vv[j]); }
         if (g0 + ATT_G < ke) issue(g0 + ATT_G);
-        KG_PROBE(25);
         float v[ATT_G * ATT_RB];
 #pragma unroll
         for (int j = 0; j < ATT_G; ++j) {
@@ -1120,7 +1106,6 @@ __device__ __forceinline__ void att_warp_slice(const Dev& D, const AttArgs& a, i
         psum += __shfl_xor_sync(0xffffffffu, psum, 16);
         l_lane = l_lane * cf + psum;
         m_lane = mn;
-        KG_PROBE(26);
         __syncwarp();
         pbuf[lane] = p;
         if (jl == 0) pbuf[32 + rl] = cf;
@@ -1221,7 +1206,6 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
     float* qs = reinterpret_cast<float*>(c.smem + WORK_OFF);       // [M_MAX][HD_MAX]
     float* mb = qs + M_MAX * HD_MAX;                               // [NWARPS][ATT_RB][ATT_MB_STRIDE]
     float* pbuf = mb + NWARPS * ATT_RB * ATT_MB_STRIDE + warp * 40;      // [NWARPS][40] probabilities of a key group
-    KG_PROBE(20);
 
     for (int item = c.cta; item < H * S; item += c.nctas) {
         const int hh = item / S, s = item % S;
@@ -1253,7 +1237,6 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
             }
         }
         cta_sync();
-        KG_PROBE(21);
         // this warp's slice of the item's keys, in whole groups
         const int nkeys = ke - kb;
         const int per = ((nkeys + NWARPS - 1) / NWARPS + ATT_G - 1) / ATT_G * ATT_G;
@@ -1262,7 +1245,6 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
             const int nr = min(ATT_RB, M - i0);
             float m_lane, l_lane, o[ATT_RB][DPL];
             att_warp_slice<WT, DPL>(D, a, hh, i0, nr, wb, we, qs, pbuf, m_lane, l_lane, o);
-            KG_PROBE(22);
 #pragma unroll
             for (int r = 0; r < ATT_RB; ++r) {
                 float* row = mb + ((size_t)warp * ATT_RB + r) * ATT_MB_STRIDE;
@@ -1300,7 +1282,6 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
                 }
             }
             cta_sync();
-            KG_PROBE(23);
         }
         if (S > 1) {
             __threadfence();
@@ -1322,9 +1303,316 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
     }
 }
 
+
+// ---- tensor-core attention (bf16 cache, head_dim 64 or 128) ----------------------------------------------------
+//
+// One pass over the keys for all rows of the pass.  A warp owns whole tiles of 16 keys and one group of 8 rows
+// (with more than 8 rows, two warps take the same tiles, one row group each: the tile's second reader finds it in
+// L2, so K and V still leave HBM once).  Everything a tile needs travels global memory -> registers -> tensor core:
+//   S = K Q^T   m16n8k16, keys on the M side, rows on the N side.  A lane loads 16 bytes (8 dims) of two key rows;
+//               which dims sit at which k position of the instruction does not matter for a dot product as long as
+//               the Q fragment (read from shared memory, rotated, pre-scaled, split into bf16 hi + lo) uses the same
+//               assignment, so no transposition is needed.
+//   online softmax in the log2 domain on the accumulator fragment (a lane holds 2 keys x 2 rows; the row maximum is
+//               a butterfly over the 8 lanes that share the rows; the row sum is reduced once, at the end).
+//   O^T = V^T P^T   m16n8k16, dims on the M side, keys on the contraction side.  A lane loads 16 bytes of four key
+//               rows and pairs equal dims of two keys with byte permutes; P (bf16 hi + lo) moves from the accumulator
+//               layout into the B layout with movmatrix.  The M position -> key assignment of the first product is
+//               chosen so that this transposition lands every key where the permuted V fragment expects it.
+// The next tile's loads are issued before the current tile is computed.
+__device__ __forceinline__ unsigned movmatrix_trans(unsigned a) {
+    unsigned d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_bf16_16816r(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int HD> struct AttTile {          // raw K / V bits of one tile as this lane holds them
+    uint4 k[2][HD / 32];                    // key rows mu(g), mu(g) + 2; 8 dims per 32-dim block
+    uint4 v[4][HD / 64];                    // key rows 4t .. 4t+3; 8 dims per 64-dim block
+};
+
+constexpr int ATT_TK = 16;                  // keys per tile
+template <int HD> struct AttSm {
+    static constexpr int QS = HD * 2 + 64;                      // bytes per Q row (padded: two rows per shared-memory phase)
+    static constexpr int Q_BYTES = 2 * M_MAX * QS;              // hi plane, lo plane
+    static constexpr int MB_OFF = (Q_BYTES + 15) / 16 * 16;     // merge buffer [NWARPS][ATT_RB][ATT_MB_STRIDE] floats
+};
+
+template <int HD>
+__device__ __forceinline__ void att_tile_load(AttTile<HD>& tl, const __nv_bfloat16* kc, const __nv_bfloat16* vc, const int* page_table,
+                                              int n_pages, int H, int hh, int psh, int psm, int key0, int last_key) {
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int mu = 4 * (g >> 1) + (g & 1);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int key = min(key0 + mu + 2 * r, last_key);
+        const int pg = __ldg(page_table + min(key >> psh, n_pages - 1));
+        const __nv_bfloat16* row = kc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + 8 * t;
+#pragma unroll
+        for (int j = 0; j < HD / 32; ++j) tl.k[r][j] = __ldcg(reinterpret_cast<const uint4*>(row + 32 * j));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int key = min(key0 + 4 * t + i, last_key);
+        const int pg = __ldg(page_table + min(key >> psh, n_pages - 1));
+        const __nv_bfloat16* row = vc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + 8 * g;
+#pragma unroll
+        for (int u = 0; u < HD / 64; ++u) tl.v[i][u] = __ldcg(reinterpret_cast<const uint4*>(row + 64 * u));
+    }
+}
+
+// Per-warp running state of one row group: lane (g, t) tracks rows 2t, 2t+1 of the group.
+template <int HD> struct AttAcc {
+    float o[HD / 16][4];      // O^T tile e: [0],[1]: dim d(e), rows 2t, 2t+1; [2],[3]: dim d(e) + 1, same rows
+    float m[2], l[2];         // running maximum (log2 domain) and this lane's share of the running sum
+};
+
+template <int HD>
+__device__ __forceinline__ void att_tile_compute(const AttTile<HD>& tl, AttAcc<HD>& ac, const unsigned char* qs, int row0, int key0,
+                                                 int ke, int pos0) {
+    // qs: shared-memory Q planes; row0: first row of this warp's row group; keys >= ke and keys a row may not see are masked
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int mu = 4 * (g >> 1) + (g & 1);
+    constexpr int QS = AttSm<HD>::QS;
+    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    const unsigned char* qh = qs + (size_t)(row0 + g) * QS + 16 * t;
+    const unsigned char* ql = qh + (size_t)M_MAX * QS;
+#pragma unroll
+    for (int j = 0; j < HD / 32; ++j) {
+        const uint4 h = *reinterpret_cast<const uint4*>(qh + 64 * j);
+        const uint4 l = *reinterpret_cast<const uint4*>(ql + 64 * j);
+        mma_bf16_16816r(sc, tl.k[0][j].x, tl.k[1][j].x, tl.k[0][j].y, tl.k[1][j].y, h.x, h.y);
+        mma_bf16_16816r(sc, tl.k[0][j].x, tl.k[1][j].x, tl.k[0][j].y, tl.k[1][j].y, l.x, l.y);
+        mma_bf16_16816r(sc, tl.k[0][j].z, tl.k[1][j].z, tl.k[0][j].w, tl.k[1][j].w, h.z, h.w);
+        mma_bf16_16816r(sc, tl.k[0][j].z, tl.k[1][j].z, tl.k[0][j].w, tl.k[1][j].w, l.z, l.w);
+    }
+    // sc[0], sc[1]: key key0 + mu, rows 2t, 2t+1;  sc[2], sc[3]: key key0 + mu + 2
+    const int ka = key0 + mu, kb2 = ka + 2;
+    const int lim0 = pos0 + row0 + 2 * t, lim1 = lim0 + 1;            // last key rows 2t / 2t+1 may see
+    if (ka >= ke || ka > lim0) sc[0] = -INFINITY;
+    if (ka >= ke || ka > lim1) sc[1] = -INFINITY;
+    if (kb2 >= ke || kb2 > lim0) sc[2] = -INFINITY;
+    if (kb2 >= ke || kb2 > lim1) sc[3] = -INFINITY;
+    float p[4];
+    float cf[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        float mx = fmaxf(sc[r], sc[2 + r]);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        const float mn = fmaxf(ac.m[r], mx);
+        cf[r] = (ac.m[r] == -INFINITY) ? 0.f : ex2f(ac.m[r] - mn);
+        p[r] = (sc[r] == -INFINITY) ? 0.f : ex2f(sc[r] - mn);
+        p[2 + r] = (sc[2 + r] == -INFINITY) ? 0.f : ex2f(sc[2 + r] - mn);
+        ac.l[r] = ac.l[r] * cf[r] + (p[r] + p[2 + r]);
+        ac.m[r] = mn;
+    }
+    // P as bf16 hi + lo, moved into the B layout: b0 = keys 4t, 4t+1 of row g; b1 = keys 4t+2, 4t+3
+    unsigned bh[2], bl[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        unsigned hi, lo;
+        split_hi_lo(make_float2(p[2 * q], p[2 * q + 1]), hi, lo);
+        bh[q] = movmatrix_trans(hi);
+        bl[q] = movmatrix_trans(lo);
+    }
+#pragma unroll
+    for (int u = 0; u < HD / 64; ++u) {
+        const unsigned w0[4] = {tl.v[0][u].x, tl.v[0][u].y, tl.v[0][u].z, tl.v[0][u].w};
+        const unsigned w1[4] = {tl.v[1][u].x, tl.v[1][u].y, tl.v[1][u].z, tl.v[1][u].w};
+        const unsigned w2[4] = {tl.v[2][u].x, tl.v[2][u].y, tl.v[2][u].z, tl.v[2][u].w};
+        const unsigned w3[4] = {tl.v[3][u].x, tl.v[3][u].y, tl.v[3][u].z, tl.v[3][u].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            // dims 64u + 8g + 2e (M rows 0-7 of the instruction) and + 1 (M rows 8-15); keys (4t, 4t+1) then (4t+2, 4t+3)
+            const unsigned a0 = __byte_perm(w0[e], w1[e], 0x5410), a1 = __byte_perm(w0[e], w1[e], 0x7632);
+            const unsigned a2 = __byte_perm(w2[e], w3[e], 0x5410), a3 = __byte_perm(w2[e], w3[e], 0x7632);
+            float (&o)[4] = ac.o[u * 4 + e];
+            o[0] *= cf[0]; o[1] *= cf[1]; o[2] *= cf[0]; o[3] *= cf[1];
+            mma_bf16_16816r(o, a0, a1, a2, a3, bh[0], bh[1]);
+            mma_bf16_16816r(o, a0, a1, a2, a3, bl[0], bl[1]);
+        }
+    }
+}
+
+template <int HD>
+__device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& c) {
+    typedef __nv_bfloat16 WT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int H = D.dm.H, d = D.dm.d, ps = D.dm.page_size, psh = D.dm.ps_shift, psm = ps - 1;
+    const int M = a.M, pos0 = a.pos0;
+    const int T = pos0 + M;
+    constexpr int half = HD / 2;
+    const int ntiles_all = (T + ATT_TK - 1) / ATT_TK;
+    // KV splits per head: the count that leaves the fewest tiles on the busiest CTA, with a fixed cost per item
+    int S = 1;
+    {
+        const float inv_ctas = 1.0f / (float)c.nctas;
+        float best = -1.f;
+#pragma unroll
+        for (int sc = 1; sc <= S_CAP; ++sc) {
+            const int chunk_ = (ntiles_all + sc - 1) / sc;
+            const float waves = ceilf((float)(H * sc) * inv_ctas - 1e-4f);
+            const float cost = waves * (float)(chunk_ + 4);
+            if ((sc == 1 || chunk_ >= 2) && (best < 0.f || cost < best)) { best = cost; S = sc; }
+        }
+    }
+    const int chunk_tiles = (ntiles_all + S - 1) / S;
+    const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;      // 1/sqrt(hd) and log2(e)
+    WT* kc = reinterpret_cast<WT*>(a.kc);
+    WT* vc = reinterpret_cast<WT*>(a.vc);
+    unsigned char* qs = reinterpret_cast<unsigned char*>(c.smem + WORK_OFF);
+    float* mb = reinterpret_cast<float*>(c.smem + WORK_OFF + AttSm<HD>::MB_OFF);
+    constexpr int QS = AttSm<HD>::QS;
+    const int R = (M + 7) >> 3;                       // row groups of 8
+    const int rg = warp % R, tlane = warp / R, tstride = NWARPS / R;
+    const int row0 = rg * 8;
+
+    for (int item = c.cta; item < H * S; item += c.nctas) {
+        const int hh = item / S, s = item % S;
+        const int tb = s * chunk_tiles, te = min(ntiles_all, tb + chunk_tiles);
+        const int kb = tb * ATT_TK, ke = min(T, te * ATT_TK);
+        AttTile<HD> t0, t1;
+        AttAcc<HD> ac;
+#pragma unroll
+        for (int e = 0; e < HD / 16; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
+        ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
+        int tile = tb + tlane;
+        // a first tile made of old keys only can be requested before this pass's K / V rows are in the cache
+        const bool early = tile < te && (tile + 1) * ATT_TK <= pos0;
+        if (early) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, tile * ATT_TK, T - 1);
+        // q rows: RoPE, scaled, split into bf16 hi + lo planes (rows >= M are zero)
+        for (int idx = tid; idx < M_MAX * half; idx += NTHREADS) {
+            const int i = idx / half, e = idx % half;
+            float r1 = 0.f, r2 = 0.f;
+            if (i < M) {
+                const float x1 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * HD + e);
+                const float x2 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * HD + e + half);
+                float cs, sn; rope_cs(D, pos0 + i, e, cs, sn);
+                r1 = (x1 * cs - x2 * sn) * qscale;
+                r2 = (x2 * cs + x1 * sn) * qscale;
+            }
+            const __nv_bfloat16 h1 = __float2bfloat16_rn(r1), h2 = __float2bfloat16_rn(r2);
+            __nv_bfloat16* ph = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)i * QS);
+            __nv_bfloat16* pl = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)(M_MAX + i) * QS);
+            ph[e] = h1; ph[e + half] = h2;
+            pl[e] = __float2bfloat16_rn(r1 - __bfloat162float(h1)); pl[e + half] = __float2bfloat16_rn(r2 - __bfloat162float(h2));
+        }
+        // append this pass's K / V rows that fall into my key range
+        {
+            const int nb = max(kb, pos0), ne = ke;
+            for (int idx = tid; idx < (ne - nb) * half; idx += NTHREADS) {
+                const int pos = nb + idx / half, e = idx % half, i = pos - pos0;
+                const float* src = a.qkv + (size_t)i * 3 * d + hh * HD;
+                const float k1 = ldcg_f(src + d + e), k2 = ldcg_f(src + d + e + half);
+                const float v1 = ldcg_f(src + 2 * d + e), v2 = ldcg_f(src + 2 * d + e + half);
+                const int page = __ldg(D.page_table + (pos >> psh));
+                float cs, sn; rope_cs(D, pos, e, cs, sn);
+                const size_t base = ((((size_t)page * H + hh) << psh) + (pos & psm)) * HD;
+                kc[base + e] = __float2bfloat16_rn(k1 * cs - k2 * sn);
+                kc[base + e + half] = __float2bfloat16_rn(k2 * cs + k1 * sn);
+                vc[base + e] = __float2bfloat16_rn(v1);
+                vc[base + e + half] = __float2bfloat16_rn(v2);
+            }
+        }
+        cta_sync();
+        if (!early && tile < te) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, tile * ATT_TK, T - 1);
+        while (tile < te) {
+            int nxt = tile + tstride;
+            if (nxt < te) att_tile_load<HD>(t1, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, nxt * ATT_TK, T - 1);
+            att_tile_compute<HD>(t0, ac, qs, row0, tile * ATT_TK, ke, pos0);
+            tile = nxt;
+            if (tile >= te) break;
+            nxt = tile + tstride;
+            if (nxt < te) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, nxt * ATT_TK, T - 1);
+            att_tile_compute<HD>(t1, ac, qs, row0, tile * ATT_TK, ke, pos0);
+            tile = nxt;
+        }
+        // the row sums: lanes that share rows add their shares in a fixed order
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 4);
+            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 8);
+            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 16);
+        }
+        // merge the warps of a row group through shared memory, four rows at a time
+        for (int rb = 0; rb * ATT_RB < M; ++rb) {
+            const int nr = min(ATT_RB, M - rb * ATT_RB);
+            if (rg == (rb >> 1) && (t >> 1) == (rb & 1)) {
+                const int rl = 2 * (t & 1);
+                float* r0 = mb + ((size_t)tlane * ATT_RB + rl) * ATT_MB_STRIDE;
+                float* r1 = r0 + ATT_MB_STRIDE;
+#pragma unroll
+                for (int e = 0; e < HD / 16; ++e) {
+                    const int dd = 64 * (e >> 2) + 8 * g + 2 * (e & 3);
+                    *reinterpret_cast<float2*>(r0 + dd) = make_float2(ac.o[e][0], ac.o[e][2]);
+                    *reinterpret_cast<float2*>(r1 + dd) = make_float2(ac.o[e][1], ac.o[e][3]);
+                }
+                if (g == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
+            }
+            cta_sync();
+            for (int idx = tid; idx < nr * HD; idx += NTHREADS) {
+                const int r = idx / HD, e = idx % HD, i = rb * ATT_RB + r;
+                float mx = -INFINITY;
+                for (int w = 0; w < tstride; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
+                float den = 0.f, num = 0.f;
+                for (int w = 0; w < tstride; ++w) {
+                    const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
+                    const float mw = row[HD_MAX];
+                    if (mw != -INFINITY) {
+                        const float wgt = ex2f(mw - mx);
+                        den += row[HD_MAX + 1] * wgt;
+                        num += row[e] * wgt;
+                    }
+                }
+                if (S == 1) {
+                    const float ov = num / den;
+                    a.out[(size_t)i * d + hh * HD + e] = ov;
+                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * HD + e, ov);
+                } else {
+                    D.att_po[(((size_t)i * H + hh) * S_CAP + s) * HD + e] = num;
+                    if (e == 0) {
+                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 0] = mx;
+                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 1] = den;
+                    }
+                }
+            }
+            cta_sync();
+        }
+        if (S > 1) {
+            __threadfence();
+            cta_sync();
+            if (tid == 0) {
+                const unsigned prev = atomicAdd(D.att_cnt + hh, 1u);
+                const int last = (prev == (unsigned)(S - 1));
+                c.ctl->att_last = last;
+                if (last) { D.att_cnt[hh] = 0u; __threadfence(); }
+            }
+            cta_sync();
+            if (*(volatile int*)&c.ctl->att_last) {
+                if (S <= 4) att_merge_splits<4, 4>(D, a, hh, S, M);
+                else if (S <= 8) att_merge_splits<8, 2>(D, a, hh, S, M);
+                else att_merge_splits<S_CAP, 1>(D, a, hh, S, M);
+            }
+            cta_sync();
+        }
+    }
+}
+static_assert(AttSm<HD_MAX>::MB_OFF + NWARPS * ATT_RB * ATT_MB_STRIDE * 4 <= WORK_BYTES, "tensor-core attention buffers do not fit in the work area");
+
 template <typename WT>
 __device__ __forceinline__ void attention_op(const Dev& D, const AttArgs* sa, Ctx& c) {
     // sa points into the consumers' operator table in shared memory
+    if constexpr (sizeof(WT) == 2) {
+        if (D.dm.hd == 128) { attention_mma<128>(D, *sa, c); return; }
+        if (D.dm.hd == 64) { attention_mma<64>(D, *sa, c); return; }
+    }
     if (D.dm.hd == 128) attention_impl<WT, 4>(D, *sa, c);
     else if (D.dm.hd == 64) attention_impl<WT, 2>(D, *sa, c);
     else attention_impl<WT, 1>(D, *sa, c);

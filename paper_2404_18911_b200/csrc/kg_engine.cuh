@@ -21,6 +21,8 @@ struct Program {
     int n;              // PREFILL: prompt length; DECODE / AR: total tokens wanted (x_0 included)
     float eta; int gamma; int stop_mode;
     int force_simple;   // 1: route bf16 linears through the plain path (cross-check)
+    unsigned long long wait_clk;   // clocks after which a device-side wait gives up (KG_E_TIMEOUT)
+    int skip_arrival;   // test hook: 1 + index of a CTA that leaves out its first grid-barrier arrival, so that a wait expires
 };
 
 #define KG_SYNC(where) do { if (!sync(where)) return false; } while (0)
@@ -63,6 +65,10 @@ struct Engine {
     // norm gain of whatever reads the output of layer i: the next layer, or the LM head after the last one
     __device__ __forceinline__ const float* next_gain(int i) const { return i + 1 < D.dm.L ? D.layers[i + 1].g1 : D.g_final; }
 
+    // an id outside [0, V) never indexes the embedding table (ids that arrive in device memory are checked by a
+    // kernel of their own, which records the error; here the access is merely kept in bounds)
+    __device__ __forceinline__ int safe_token(int tok) const { return (unsigned)tok < (unsigned)D.dm.V ? tok : 0; }
+
     // h[i] = E[token_i]; packed for layer 0
     __device__ void embed_rows(const int* toks_global, int tok_single, int M) {
         if (c.producer) return;
@@ -71,7 +77,7 @@ struct Engine {
         if (!streamed()) {
             for (int idx = c.cta * NTHREADS + threadIdx.x; idx < M * d; idx += c.nctas * NTHREADS) {
                 const int i = idx / d, e = idx % d;
-                const int tok = toks_global ? __ldcg(toks_global + i) : tok_single;
+                const int tok = safe_token(toks_global ? __ldcg(toks_global + i) : tok_single);
                 D.h[idx] = wt_to_float<WT>(E[(size_t)tok * d + e]);
             }
             return;
@@ -80,7 +86,7 @@ struct Engine {
         a.N = d; a.M = M; a.out = D.h; a.ldo = d;
         a.pk[0] = PkOut{D.layers[0].g1, D.hA_pk}; a.ldpk_out = (int)ldpk(); a.ssq_out = D.ssq_hA;
         emit_plain_rows(a, c, [&](int m, int e) {
-            const int tok = toks_global ? __ldcg(toks_global + m) : tok_single;
+            const int tok = safe_token(toks_global ? __ldcg(toks_global + m) : tok_single);
             return wt_to_float<WT>(E[(size_t)tok * d + e]);
         });
     }
@@ -377,6 +383,8 @@ struct Engine {
     }
 
     __device__ void run() {
+        // the plain path streams nothing: its producer warp has no part in the launch
+        if (c.producer && !streamed()) return;
         load_state();
         const bool ok = run_program();
         if (!ok && c.producer) ring_drain(c);
@@ -386,7 +394,7 @@ struct Engine {
 template <typename WT>
 __global__ void __launch_bounds__(BLOCK_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
     extern __shared__ __align__(128) char smem[];
-    Ctx& c = ctx_init(smem, D.st, D.bar, true);
+    Ctx& c = ctx_init(smem, D.st, D.bar, true, pg.wait_clk, pg.skip_arrival);
     Engine<WT> eng(D, c, pg);
     eng.run();
 }
