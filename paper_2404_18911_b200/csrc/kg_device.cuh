@@ -1306,20 +1306,22 @@ __device__ __noinline__ void attention_impl(const Dev& D, const AttArgs& a, Ctx&
 
 // ---- tensor-core attention (bf16 cache, head_dim 64 or 128) ----------------------------------------------------
 //
-// One pass over the keys for all rows of the pass.  A warp owns whole tiles of 16 keys and one group of 8 rows
-// (with more than 8 rows, two warps take the same tiles, one row group each: the tile's second reader finds it in
-// L2, so K and V still leave HBM once).  Everything a tile needs travels global memory -> registers -> tensor core:
+// One pass over the keys for all rows of the pass.  The unit of work is a tile of 16 keys and one group of 8 rows
+// (with more than 8 rows, two units take the same tiles, one row group each: the tile's second reader finds it in
+// L2, so K and V still leave HBM once).  A unit is one warp when head_dim is 64; with head_dim 128 it is a pair of
+// warps that own 64 dims each, which keeps a warp's share of K, V and the output small enough to hold two tiles in
+// registers.  Everything a tile needs travels global memory -> registers -> tensor core:
 //   S = K Q^T   m16n8k16, keys on the M side, rows on the N side.  A lane loads 16 bytes (8 dims) of two key rows;
 //               which dims sit at which k position of the instruction does not matter for a dot product as long as
 //               the Q fragment (read from shared memory, rotated, pre-scaled, split into bf16 hi + lo) uses the same
-//               assignment, so no transposition is needed.
+//               assignment, so no transposition is needed.  The two warps of a pair add their halves of the dot
+//               products through shared memory (one named barrier per tile); both then hold the same scores.
 //   online softmax in the log2 domain on the accumulator fragment (a lane holds 2 keys x 2 rows; the row maximum is
 //               a butterfly over the 8 lanes that share the rows; the row sum is reduced once, at the end).
 //   O^T = V^T P^T   m16n8k16, dims on the M side, keys on the contraction side.  A lane loads 16 bytes of four key
 //               rows and pairs equal dims of two keys with byte permutes; P (bf16 hi + lo) moves from the accumulator
 //               layout into the B layout with movmatrix.  The M position -> key assignment of the first product is
 //               chosen so that this transposition lands every key where the permuted V fragment expects it.
-// The next tile's loads are issued before the current tile is computed.
 __device__ __forceinline__ unsigned movmatrix_trans(unsigned a) {
     unsigned d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -1329,76 +1331,90 @@ __device__ __forceinline__ void mma_bf16_16816r(float (&c)[4], unsigned a0, unsi
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-template <int HD> struct AttTile {          // raw K / V bits of one tile as this lane holds them
-    uint4 k[2][HD / 32];                    // key rows mu(g), mu(g) + 2; 8 dims per 32-dim block
-    uint4 v[4][HD / 64];                    // key rows 4t .. 4t+3; 8 dims per 64-dim block
-};
+// barrier among the two warps of a pair (ids 2 .. 5; 0 is the whole CTA, 1 the consumer warps)
+__device__ __forceinline__ void pair_sync(int pair) { asm volatile("bar.sync %0, 64;" ::"r"(2 + pair) : "memory"); }
 
 constexpr int ATT_TK = 16;                  // keys per tile
+constexpr int ATT_DW = 64;                  // dims per warp
+struct AttK { uint4 k[2][2]; };             // raw K bits of a tile: key rows mu(g), mu(g) + 2; 8 dims of each 32-dim block
+struct AttV { uint4 v[4]; };                // raw V bits of a tile: key rows 4t .. 4t+3; dims 8g .. 8g+7 of the warp's 64
+struct AttAcc {                             // running state of a unit's rows: lane (g, t) tracks rows 2t, 2t+1
+    float o[4][4];                          // O^T tile e: [0],[1]: dim 8g + 2e, rows 2t, 2t+1; [2],[3]: dim 8g + 2e + 1
+    float m[2], l[2];                       // running maximum (log2 domain) and this lane's share of the running sum
+};
+struct AttP { unsigned bh[2], bl[2]; float cf[2]; };    // a tile's probabilities in the B layout (bf16 hi, lo), rescale factors
+
 template <int HD> struct AttSm {
     static constexpr int QS = HD * 2 + 64;                      // bytes per Q row (padded: two rows per shared-memory phase)
     static constexpr int Q_BYTES = 2 * M_MAX * QS;              // hi plane, lo plane
-    static constexpr int MB_OFF = (Q_BYTES + 15) / 16 * 16;     // merge buffer [NWARPS][ATT_RB][ATT_MB_STRIDE] floats
+    static constexpr int MB_OFF = (Q_BYTES + 15) / 16 * 16;     // merge buffer [units][ATT_RB][ATT_MB_STRIDE] floats; while the
+                                                                // tiles run, the pairs' score exchange [4][2][2][32] float4
 };
 
+// Page-table entries of a window of 32 pages, one per lane; a lane asks for the page of a key by shuffle.
+struct PageWin {
+    int first, pgs;
+    __device__ __forceinline__ void load(const int* page_table, int n_pages, int first_page) {
+        first = first_page;
+        pgs = __ldg(page_table + min(first_page + (int)(threadIdx.x & 31), n_pages - 1));
+    }
+    // every lane calls this with its own key; the keys of one call lie within [first, first + 32) pages
+    __device__ __forceinline__ int page_of(int key, int psh) const { return __shfl_sync(0xffffffffu, pgs, (key >> psh) - first); }
+};
+
+// kc / vc point at the warp's first dim of the head (element offset hh * HD + dim offset is added by the caller per row)
 template <int HD>
-__device__ __forceinline__ void att_tile_load(AttTile<HD>& tl, const __nv_bfloat16* kc, const __nv_bfloat16* vc, const int* page_table,
-                                              int n_pages, int H, int hh, int psh, int psm, int key0, int last_key) {
+__device__ __forceinline__ void att_load(AttK& tk, AttV& tv, const __nv_bfloat16* kc, const __nv_bfloat16* vc, const PageWin& pw,
+                                         int H, int hh, int dof, int psh, int psm, int key0, int last_key) {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int mu = 4 * (g >> 1) + (g & 1);
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int key = min(key0 + mu + 2 * r, last_key);
-        const int pg = __ldg(page_table + min(key >> psh, n_pages - 1));
-        const __nv_bfloat16* row = kc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + 8 * t;
-#pragma unroll
-        for (int j = 0; j < HD / 32; ++j) tl.k[r][j] = __ldcg(reinterpret_cast<const uint4*>(row + 32 * j));
+        const int pg = pw.page_of(key, psh);
+        const __nv_bfloat16* row = kc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + dof + 8 * t;
+        tk.k[r][0] = __ldcg(reinterpret_cast<const uint4*>(row));
+        tk.k[r][1] = __ldcg(reinterpret_cast<const uint4*>(row + 32));
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int key = min(key0 + 4 * t + i, last_key);
-        const int pg = __ldg(page_table + min(key >> psh, n_pages - 1));
-        const __nv_bfloat16* row = vc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + 8 * g;
-#pragma unroll
-        for (int u = 0; u < HD / 64; ++u) tl.v[i][u] = __ldcg(reinterpret_cast<const uint4*>(row + 64 * u));
+        const int pg = pw.page_of(key, psh);
+        const __nv_bfloat16* row = vc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + dof + 8 * g;
+        tv.v[i] = __ldcg(reinterpret_cast<const uint4*>(row));
     }
 }
 
-// Per-warp running state of one row group: lane (g, t) tracks rows 2t, 2t+1 of the group.
-template <int HD> struct AttAcc {
-    float o[HD / 16][4];      // O^T tile e: [0],[1]: dim d(e), rows 2t, 2t+1; [2],[3]: dim d(e) + 1, same rows
-    float m[2], l[2];         // running maximum (log2 domain) and this lane's share of the running sum
-};
-
-template <int HD>
-__device__ __forceinline__ void att_tile_compute(const AttTile<HD>& tl, AttAcc<HD>& ac, const unsigned char* qs, int row0, int key0,
-                                                 int ke, int pos0) {
-    // qs: shared-memory Q planes; row0: first row of this warp's row group; keys >= ke and keys a row may not see are masked
+// This warp's 64 dims of S = K Q^T for one tile: sc[0], sc[1]: key key0 + mu(g), rows 2t, 2t+1; sc[2], sc[3]: key + 2.
+// qw: shared-memory address of the hi plane at this warp's first dim; row stride QS, lo plane M_MAX rows further.
+template <int QS>
+__device__ __forceinline__ void att_scores(const AttK& tk, float (&sc)[4], uint32_t qw, int row0) {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const int mu = 4 * (g >> 1) + (g & 1);
-    constexpr int QS = AttSm<HD>::QS;
-    float sc[4] = {0.f, 0.f, 0.f, 0.f};
-    const unsigned char* qh = qs + (size_t)(row0 + g) * QS + 16 * t;
-    const unsigned char* ql = qh + (size_t)M_MAX * QS;
+    const uint32_t qh = qw + (uint32_t)((row0 + g) * QS + 16 * t);
+    const uint32_t ql = qh + (uint32_t)(M_MAX * QS);
+    sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
 #pragma unroll
-    for (int j = 0; j < HD / 32; ++j) {
-        const uint4 h = *reinterpret_cast<const uint4*>(qh + 64 * j);
-        const uint4 l = *reinterpret_cast<const uint4*>(ql + 64 * j);
-        mma_bf16_16816r(sc, tl.k[0][j].x, tl.k[1][j].x, tl.k[0][j].y, tl.k[1][j].y, h.x, h.y);
-        mma_bf16_16816r(sc, tl.k[0][j].x, tl.k[1][j].x, tl.k[0][j].y, tl.k[1][j].y, l.x, l.y);
-        mma_bf16_16816r(sc, tl.k[0][j].z, tl.k[1][j].z, tl.k[0][j].w, tl.k[1][j].w, h.z, h.w);
-        mma_bf16_16816r(sc, tl.k[0][j].z, tl.k[1][j].z, tl.k[0][j].w, tl.k[1][j].w, l.z, l.w);
+    for (int j = 0; j < 2; ++j) {
+        uint4 h, l;
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(h.x), "=r"(h.y), "=r"(h.z), "=r"(h.w) : "r"(qh + 64u * j));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(l.x), "=r"(l.y), "=r"(l.z), "=r"(l.w) : "r"(ql + 64u * j));
+        mma_bf16_16816r(sc, tk.k[0][j].x, tk.k[1][j].x, tk.k[0][j].y, tk.k[1][j].y, h.x, h.y);
+        mma_bf16_16816r(sc, tk.k[0][j].x, tk.k[1][j].x, tk.k[0][j].y, tk.k[1][j].y, l.x, l.y);
+        mma_bf16_16816r(sc, tk.k[0][j].z, tk.k[1][j].z, tk.k[0][j].w, tk.k[1][j].w, h.z, h.w);
+        mma_bf16_16816r(sc, tk.k[0][j].z, tk.k[1][j].z, tk.k[0][j].w, tk.k[1][j].w, l.z, l.w);
     }
-    // sc[0], sc[1]: key key0 + mu, rows 2t, 2t+1;  sc[2], sc[3]: key key0 + mu + 2
-    const int ka = key0 + mu, kb2 = ka + 2;
+}
+
+// Masking, online-softmax update and the probabilities of a tile in the layout the second product reads.
+__device__ __forceinline__ void att_softmax(float (&sc)[4], AttAcc& ac, AttP& pp, int row0, int key0, int ke, int pos0) {
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int ka = key0 + 4 * (g >> 1) + (g & 1), kb2 = ka + 2;
     const int lim0 = pos0 + row0 + 2 * t, lim1 = lim0 + 1;            // last key rows 2t / 2t+1 may see
     if (ka >= ke || ka > lim0) sc[0] = -INFINITY;
     if (ka >= ke || ka > lim1) sc[1] = -INFINITY;
     if (kb2 >= ke || kb2 > lim0) sc[2] = -INFINITY;
     if (kb2 >= ke || kb2 > lim1) sc[3] = -INFINITY;
     float p[4];
-    float cf[2];
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         float mx = fmaxf(sc[r], sc[2 + r]);
@@ -1406,51 +1422,58 @@ __device__ __forceinline__ void att_tile_compute(const AttTile<HD>& tl, AttAcc<H
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
         const float mn = fmaxf(ac.m[r], mx);
-        cf[r] = (ac.m[r] == -INFINITY) ? 0.f : ex2f(ac.m[r] - mn);
+        pp.cf[r] = (ac.m[r] == -INFINITY) ? 0.f : ex2f(ac.m[r] - mn);
         p[r] = (sc[r] == -INFINITY) ? 0.f : ex2f(sc[r] - mn);
         p[2 + r] = (sc[2 + r] == -INFINITY) ? 0.f : ex2f(sc[2 + r] - mn);
-        ac.l[r] = ac.l[r] * cf[r] + (p[r] + p[2 + r]);
+        ac.l[r] = ac.l[r] * pp.cf[r] + (p[r] + p[2 + r]);
         ac.m[r] = mn;
     }
     // P as bf16 hi + lo, moved into the B layout: b0 = keys 4t, 4t+1 of row g; b1 = keys 4t+2, 4t+3
-    unsigned bh[2], bl[2];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
         unsigned hi, lo;
         split_hi_lo(make_float2(p[2 * q], p[2 * q + 1]), hi, lo);
-        bh[q] = movmatrix_trans(hi);
-        bl[q] = movmatrix_trans(lo);
+        pp.bh[q] = movmatrix_trans(hi);
+        pp.bl[q] = movmatrix_trans(lo);
     }
+}
+
+// O^T += V^T P^T on this warp's 64 dims
+__device__ __forceinline__ void att_accumulate(const AttV& tv, AttAcc& ac, const AttP& pp) {
+    const unsigned w0[4] = {tv.v[0].x, tv.v[0].y, tv.v[0].z, tv.v[0].w};
+    const unsigned w1[4] = {tv.v[1].x, tv.v[1].y, tv.v[1].z, tv.v[1].w};
+    const unsigned w2[4] = {tv.v[2].x, tv.v[2].y, tv.v[2].z, tv.v[2].w};
+    const unsigned w3[4] = {tv.v[3].x, tv.v[3].y, tv.v[3].z, tv.v[3].w};
 #pragma unroll
-    for (int u = 0; u < HD / 64; ++u) {
-        const unsigned w0[4] = {tl.v[0][u].x, tl.v[0][u].y, tl.v[0][u].z, tl.v[0][u].w};
-        const unsigned w1[4] = {tl.v[1][u].x, tl.v[1][u].y, tl.v[1][u].z, tl.v[1][u].w};
-        const unsigned w2[4] = {tl.v[2][u].x, tl.v[2][u].y, tl.v[2][u].z, tl.v[2][u].w};
-        const unsigned w3[4] = {tl.v[3][u].x, tl.v[3][u].y, tl.v[3][u].z, tl.v[3][u].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            // dims 64u + 8g + 2e (M rows 0-7 of the instruction) and + 1 (M rows 8-15); keys (4t, 4t+1) then (4t+2, 4t+3)
-            const unsigned a0 = __byte_perm(w0[e], w1[e], 0x5410), a1 = __byte_perm(w0[e], w1[e], 0x7632);
-            const unsigned a2 = __byte_perm(w2[e], w3[e], 0x5410), a3 = __byte_perm(w2[e], w3[e], 0x7632);
-            float (&o)[4] = ac.o[u * 4 + e];
-            o[0] *= cf[0]; o[1] *= cf[1]; o[2] *= cf[0]; o[3] *= cf[1];
-            mma_bf16_16816r(o, a0, a1, a2, a3, bh[0], bh[1]);
-            mma_bf16_16816r(o, a0, a1, a2, a3, bl[0], bl[1]);
-        }
+    for (int e = 0; e < 4; ++e) {
+        // dims 8g + 2e (M rows 0-7 of the instruction) and + 1 (M rows 8-15); keys (4t, 4t+1) then (4t+2, 4t+3)
+        const unsigned a0 = __byte_perm(w0[e], w1[e], 0x5410), a1 = __byte_perm(w0[e], w1[e], 0x7632);
+        const unsigned a2 = __byte_perm(w2[e], w3[e], 0x5410), a3 = __byte_perm(w2[e], w3[e], 0x7632);
+        float (&o)[4] = ac.o[e];
+        o[0] *= pp.cf[0]; o[1] *= pp.cf[1]; o[2] *= pp.cf[0]; o[3] *= pp.cf[1];
+        mma_bf16_16816r(o, a0, a1, a2, a3, pp.bh[0], pp.bh[1]);
+        mma_bf16_16816r(o, a0, a1, a2, a3, pp.bl[0], pp.bl[1]);
     }
 }
 
 template <int HD>
 __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& c) {
     typedef __nv_bfloat16 WT;
+    constexpr int NSPLIT = HD / ATT_DW;               // warps per unit: 1 (head_dim 64) or 2 (head_dim 128)
+    constexpr int NUNITS = NWARPS / NSPLIT;
+    constexpr int half = HD / 2;
+    constexpr int QS = AttSm<HD>::QS;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const int H = D.dm.H, d = D.dm.d, ps = D.dm.page_size, psh = D.dm.ps_shift, psm = ps - 1;
+    const int H = D.dm.H, d = D.dm.d, psh = D.dm.ps_shift, psm = D.dm.page_size - 1;
     const int M = a.M, pos0 = a.pos0;
     const int T = pos0 + M;
-    constexpr int half = HD / 2;
     const int ntiles_all = (T + ATT_TK - 1) / ATT_TK;
-    // KV splits per head: the count that leaves the fewest tiles on the busiest CTA, with a fixed cost per item
+    const int R = (M + 7) >> 3;                       // row groups of 8
+    const int nw = NUNITS / R;                        // units that share the tiles of an item
+    // KV splits per head.  An item costs its units' tiles (one memory latency each) plus a fixed part, and a head
+    // that is split pays for the merge of its partials through global memory (several dependent round trips, about
+    // as long as three tiles): very short caches stay unsplit.
     int S = 1;
     {
         const float inv_ctas = 1.0f / (float)c.nctas;
@@ -1458,62 +1481,52 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
 #pragma unroll
         for (int sc = 1; sc <= S_CAP; ++sc) {
             const int chunk_ = (ntiles_all + sc - 1) / sc;
+            const int tpw_ = (chunk_ + nw - 1) / nw;
             const float waves = ceilf((float)(H * sc) * inv_ctas - 1e-4f);
-            const float cost = waves * (float)(chunk_ + 4);
+            const float cost = waves * (float)(tpw_ + 2 + (sc > 1 ? 3 : 0));
             if ((sc == 1 || chunk_ >= 2) && (best < 0.f || cost < best)) { best = cost; S = sc; }
         }
     }
     const int chunk_tiles = (ntiles_all + S - 1) / S;
+    const int tpw = (chunk_tiles + nw - 1) / nw;
     const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;      // 1/sqrt(hd) and log2(e)
     WT* kc = reinterpret_cast<WT*>(a.kc);
     WT* vc = reinterpret_cast<WT*>(a.vc);
     unsigned char* qs = reinterpret_cast<unsigned char*>(c.smem + WORK_OFF);
     float* mb = reinterpret_cast<float*>(c.smem + WORK_OFF + AttSm<HD>::MB_OFF);
-    constexpr int QS = AttSm<HD>::QS;
-    const int R = (M + 7) >> 3;                       // row groups of 8
-    const int rg = warp % R, tlane = warp / R, tstride = NWARPS / R;
+    const int unit = warp / NSPLIT, hsel = warp % NSPLIT, dof = hsel * ATT_DW;
+    const int rg = unit % R, tlane = unit / R;
     const int row0 = rg * 8;
+    const uint32_t qw = smem_u32(qs) + (uint32_t)(dof * 2);
+    // rows >= M of the row groups in use are zero in both planes
+    for (int idx = tid; idx < (8 * R - M) * half; idx += NTHREADS) {
+        const int i = M + idx / half, e = idx % half;
+        reinterpret_cast<unsigned*>(qs + (size_t)i * QS)[e] = 0u;
+        reinterpret_cast<unsigned*>(qs + (size_t)(M_MAX + i) * QS)[e] = 0u;
+    }
 
     for (int item = c.cta; item < H * S; item += c.nctas) {
         const int hh = item / S, s = item % S;
         const int tb = s * chunk_tiles, te = min(ntiles_all, tb + chunk_tiles);
         const int kb = tb * ATT_TK, ke = min(T, te * ATT_TK);
-        AttTile<HD> t0, t1;
-        AttAcc<HD> ac;
-#pragma unroll
-        for (int e = 0; e < HD / 16; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
-        ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
-        int tile = tb + tlane;
-        // a first tile made of old keys only can be requested before this pass's K / V rows are in the cache
-        const bool early = tile < te && (tile + 1) * ATT_TK <= pos0;
-        if (early) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, tile * ATT_TK, T - 1);
-        // q rows: RoPE, scaled, split into bf16 hi + lo planes (rows >= M are zero)
-        for (int idx = tid; idx < M_MAX * half; idx += NTHREADS) {
-            const int i = idx / half, e = idx % half;
-            float r1 = 0.f, r2 = 0.f;
-            if (i < M) {
-                const float x1 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * HD + e);
-                const float x2 = ldcg_f(a.qkv + (size_t)i * 3 * d + hh * HD + e + half);
-                float cs, sn; rope_cs(D, pos0 + i, e, cs, sn);
-                r1 = (x1 * cs - x2 * sn) * qscale;
-                r2 = (x2 * cs + x1 * sn) * qscale;
-            }
+        // this pass's rows: q rotated, scaled and split into the bf16 hi / lo planes; k rotated and, with v, rounded and
+        // appended to the cache when the row's position lies in my key range.  One cos / sin pair serves q and k, and
+        // all six loads of an element are issued before the first is used.
+        for (int idx = tid; idx < M * half; idx += NTHREADS) {
+            const int i = idx / half, e = idx % half, pos = pos0 + i;
+            const float* src = a.qkv + (size_t)i * 3 * d + hh * HD + e;
+            const float q1 = ldcg_f(src), q2 = ldcg_f(src + half);
+            const float k1 = ldcg_f(src + d), k2 = ldcg_f(src + d + half);
+            const float v1 = ldcg_f(src + 2 * d), v2 = ldcg_f(src + 2 * d + half);
+            const int page = __ldg(D.page_table + (pos >> psh));
+            float cs, sn; rope_cs(D, pos, e, cs, sn);
+            const float r1 = (q1 * cs - q2 * sn) * qscale, r2 = (q2 * cs + q1 * sn) * qscale;
             const __nv_bfloat16 h1 = __float2bfloat16_rn(r1), h2 = __float2bfloat16_rn(r2);
             __nv_bfloat16* ph = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)i * QS);
             __nv_bfloat16* pl = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)(M_MAX + i) * QS);
             ph[e] = h1; ph[e + half] = h2;
             pl[e] = __float2bfloat16_rn(r1 - __bfloat162float(h1)); pl[e + half] = __float2bfloat16_rn(r2 - __bfloat162float(h2));
-        }
-        // append this pass's K / V rows that fall into my key range
-        {
-            const int nb = max(kb, pos0), ne = ke;
-            for (int idx = tid; idx < (ne - nb) * half; idx += NTHREADS) {
-                const int pos = nb + idx / half, e = idx % half, i = pos - pos0;
-                const float* src = a.qkv + (size_t)i * 3 * d + hh * HD;
-                const float k1 = ldcg_f(src + d + e), k2 = ldcg_f(src + d + e + half);
-                const float v1 = ldcg_f(src + 2 * d + e), v2 = ldcg_f(src + 2 * d + e + half);
-                const int page = __ldg(D.page_table + (pos >> psh));
-                float cs, sn; rope_cs(D, pos, e, cs, sn);
+            if (pos >= kb && pos < ke) {
                 const size_t base = ((((size_t)page * H + hh) << psh) + (pos & psm)) * HD;
                 kc[base + e] = __float2bfloat16_rn(k1 * cs - k2 * sn);
                 kc[base + e + half] = __float2bfloat16_rn(k2 * cs + k1 * sn);
@@ -1521,18 +1534,45 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
                 vc[base + e + half] = __float2bfloat16_rn(v2);
             }
         }
+        AttAcc ac;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
+        ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
+        // this unit's tiles: a contiguous run, so that one window of page-table entries serves many of them
+        int tile = tb + tlane * tpw;
+        const int tend = min(te, tile + tpw);
+        PageWin pw;
+        if (tile < tend) pw.load(D.page_table, D.dm.n_pages, (tile * ATT_TK) >> psh);
         cta_sync();
-        if (!early && tile < te) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, tile * ATT_TK, T - 1);
-        while (tile < te) {
-            int nxt = tile + tstride;
-            if (nxt < te) att_tile_load<HD>(t1, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, nxt * ATT_TK, T - 1);
-            att_tile_compute<HD>(t0, ac, qs, row0, tile * ATT_TK, ke, pos0);
-            tile = nxt;
-            if (tile >= te) break;
-            nxt = tile + tstride;
-            if (nxt < te) att_tile_load<HD>(t0, kc, vc, D.page_table, D.dm.n_pages, H, hh, psh, psm, nxt * ATT_TK, T - 1);
-            att_tile_compute<HD>(t1, ac, qs, row0, tile * ATT_TK, ke, pos0);
-            tile = nxt;
+        auto fetch = [&](AttK& tk, AttV& tv, int ti) {
+            const int key0 = ti * ATT_TK, key1 = min(key0 + ATT_TK - 1, T - 1);
+            if ((key1 >> psh) - pw.first >= 32) pw.load(D.page_table, D.dm.n_pages, key0 >> psh);
+            att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1);
+        };
+        AttP pp;
+        auto step = [&](const AttK& tk, const AttV& tv, int ti) {
+            float sc[4];
+            att_scores<QS>(tk, sc, qw, row0);
+            if constexpr (NSPLIT == 2) {
+                // the pair's halves of the dot products meet in shared memory (two buffers, used alternately)
+                float4* xb = reinterpret_cast<float4*>(mb) + (size_t)((unit * 2 + (ti & 1)) * 2) * 32;
+                xb[hsel * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+                pair_sync(unit);
+                const float4 ot = xb[(hsel ^ 1) * 32 + lane];
+                sc[0] += ot.x; sc[1] += ot.y; sc[2] += ot.z; sc[3] += ot.w;
+            }
+            att_softmax(sc, ac, pp, row0, ti * ATT_TK, ke, pos0);
+            att_accumulate(tv, ac, pp);
+        };
+        // One register set for K and V (a second one would not fit: the register allocation is shared with the
+        // linear operators).  A tile therefore costs a memory latency; the split count above keeps the run of
+        // tiles per unit short, and the other units and CTAs keep the memory system busy meanwhile.
+        AttK k0;
+        AttV v0;
+        while (tile < tend) {
+            fetch(k0, v0, tile);
+            step(k0, v0, tile);
+            ++tile;
         }
         // the row sums: lanes that share rows add their shares in a fixed order
 #pragma unroll
@@ -1541,7 +1581,8 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
             ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 8);
             ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 16);
         }
-        // merge the warps of a row group through shared memory, four rows at a time
+        if constexpr (NSPLIT == 2) cta_sync();          // the merge buffer lies over the pairs' exchange buffers
+        // merge the units of a row group through shared memory, four rows at a time
         for (int rb = 0; rb * ATT_RB < M; ++rb) {
             const int nr = min(ATT_RB, M - rb * ATT_RB);
             if (rg == (rb >> 1) && (t >> 1) == (rb & 1)) {
@@ -1549,20 +1590,20 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
                 float* r0 = mb + ((size_t)tlane * ATT_RB + rl) * ATT_MB_STRIDE;
                 float* r1 = r0 + ATT_MB_STRIDE;
 #pragma unroll
-                for (int e = 0; e < HD / 16; ++e) {
-                    const int dd = 64 * (e >> 2) + 8 * g + 2 * (e & 3);
+                for (int e = 0; e < 4; ++e) {
+                    const int dd = dof + 8 * g + 2 * e;
                     *reinterpret_cast<float2*>(r0 + dd) = make_float2(ac.o[e][0], ac.o[e][2]);
                     *reinterpret_cast<float2*>(r1 + dd) = make_float2(ac.o[e][1], ac.o[e][3]);
                 }
-                if (g == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
+                if (g == 0 && hsel == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
             }
             cta_sync();
             for (int idx = tid; idx < nr * HD; idx += NTHREADS) {
                 const int r = idx / HD, e = idx % HD, i = rb * ATT_RB + r;
                 float mx = -INFINITY;
-                for (int w = 0; w < tstride; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
+                for (int w = 0; w < nw; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
                 float den = 0.f, num = 0.f;
-                for (int w = 0; w < tstride; ++w) {
+                for (int w = 0; w < nw; ++w) {
                     const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
                     const float mw = row[HD_MAX];
                     if (mw != -INFINITY) {
