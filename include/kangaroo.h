@@ -35,7 +35,9 @@ typedef enum {
     KG_E_SEQ_FULL = -4,  /* the sequence would exceed max_seq */
     KG_E_CUDA = -5,      /* a CUDA runtime call failed */
     KG_E_TIMEOUT = -6,   /* a bounded device-side wait expired; the model must be re-initialised (kg_init_model) */
-    KG_E_LIMIT = -7      /* a size exceeds what a fixed-capacity entry point (kg_op_lm_head_noalloc) can hold */
+    KG_E_LIMIT = -7,     /* a size exceeds what a fixed-capacity entry point (kg_op_lm_head_noalloc) can hold */
+    KG_E_INTERNAL = -8   /* a kernel found an index outside its table (e.g. a page number), skipped the access and
+                            recorded it; kg_last_cuda_error() says which check; the model must be re-initialised */
 } kg_status;
 
 enum { KG_F32 = 0, KG_BF16 = 1 };            /* storage type of weights and KV cache */
@@ -173,7 +175,7 @@ int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t seed);
 
 /* ---- test hooks (no part of the method; used by the parity and failure-path tests) ----------------
  * kg_debug_force_simple: route a bf16 model's linear operators through the plain (non tensor-core) path, a
- *   cross-check of the streamed path.  kg_debug_force_simple_ops: the same for the single-operator calls.
+ *   cross-check of the streamed path; KG_E_ARG for shapes whose 16 rows of max(d, F) floats do not fit in shared memory.  kg_debug_force_simple_ops: the same for the single-operator calls.
  * kg_debug_set_wait_budget: every wait inside a kernel (grid barrier, weight ring) gives up after this many
  *   milliseconds (default about 3 s) and the launch ends with KG_E_TIMEOUT in the state word.
  * kg_debug_skip_barrier_arrival: in the NEXT launch, CTA `cta` leaves out its first grid-barrier arrival, so that
@@ -228,6 +230,9 @@ int kg_op_attention(int32_t dtype, const float* qkv_dev, int32_t M, int32_t pos0
                     int32_t page_size, float* out_dev, void* scratch_dev, void* cuda_stream);
 
 const char* kg_strerror(int status);
+/* After a call of this thread returned KG_E_CUDA: which CUDA runtime call failed and the runtime's name and text
+ * for the error ("" if none failed yet).  The string is owned by the library and valid until the next failure. */
+const char* kg_last_cuda_error(void);
 
 #ifdef __cplusplus
 }

@@ -17,14 +17,14 @@ KG_GAMMA_MAX = KG_M_MAX - 1
 KG_F32, KG_BF16 = 0, 1
 STOP_KEEP, STOP_DROP = 0, 1
 
-KG_OK, KG_E_ARG, KG_E_STATE, KG_E_NOMEM, KG_E_SEQ_FULL, KG_E_CUDA, KG_E_TIMEOUT, KG_E_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7
+KG_OK, KG_E_ARG, KG_E_STATE, KG_E_NOMEM, KG_E_SEQ_FULL, KG_E_CUDA, KG_E_TIMEOUT, KG_E_LIMIT, KG_E_INTERNAL = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
     "kg_workspace_bytes", "kg_init_model", "kg_free_model", "kg_reset", "kg_prefill", "kg_prefill_device",
     "kg_draft", "kg_verify", "kg_decode", "kg_decode_ar", "kg_generate", "kg_read_tokens", "kg_read_S", "kg_read_round_log",
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
     "kg_op_lm_head", "kg_op_lm_head_noalloc", "kg_op_attention", "kg_strerror",
-    "kg_debug_force_simple", "kg_debug_force_simple_ops", "kg_debug_set_wait_budget", "kg_debug_skip_barrier_arrival",
+    "kg_last_cuda_error", "kg_debug_force_simple", "kg_debug_force_simple_ops", "kg_debug_set_wait_budget", "kg_debug_skip_barrier_arrival",
 ]
 
 
@@ -71,7 +71,10 @@ class KgStats(C.Structure):
 class KgError(RuntimeError):
     def __init__(self, status, what):
         self.status = status
-        super().__init__(f"{what}: {status} ({strerror(status)})")
+        detail = ""
+        if status in (KG_E_CUDA, KG_E_INTERNAL):
+            detail = " [" + load().kg_last_cuda_error().decode() + "]"
+        super().__init__(f"{what}: {status} ({strerror(status)}){detail}")
 
 
 _lib = None
@@ -113,6 +116,8 @@ def load():
     lib.kg_op_attention.argtypes = [i32, vp, i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, vp, vp]
     lib.kg_strerror.restype = C.c_char_p
     lib.kg_strerror.argtypes = [C.c_int]
+    lib.kg_last_cuda_error.restype = C.c_char_p
+    lib.kg_last_cuda_error.argtypes = []
     lib.kg_debug_force_simple.argtypes = [vp, C.c_int]
     lib.kg_debug_force_simple_ops.argtypes = [C.c_int]
     lib.kg_debug_set_wait_budget.argtypes = [vp, C.c_double]

@@ -234,7 +234,16 @@ struct kg_model {
     std::vector<LayerW> layers_host;
 };
 
-#define CK(x) do { if ((x) != cudaSuccess) return KG_E_CUDA; } while (0)
+// Name and text of the CUDA error behind the last KG_E_CUDA of this thread ("" if there was none).
+static thread_local char g_cuda_err[160] = "";
+static bool cuda_failed(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return false;
+    std::snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+    return true;
+}
+#define CK(x) do { if (cuda_failed((x), #x)) return KG_E_CUDA; } while (0)
+
+extern "C" const char* kg_last_cuda_error(void) { return g_cuda_err; }
 
 extern "C" const char* kg_strerror(int s) {
     switch (s) {
@@ -246,6 +255,7 @@ extern "C" const char* kg_strerror(int s) {
         case KG_E_CUDA: return "CUDA runtime error";
         case KG_E_TIMEOUT: return "device-side wait timed out";
         case KG_E_LIMIT: return "size beyond the capacity of the library's static scratch";
+        case KG_E_INTERNAL: return "a device-side index check failed (the access was skipped)";
         default: return "unknown status";
     }
 }
@@ -275,6 +285,11 @@ static int read_state(kg_model* m, State* out) {
     CK(cudaMemcpyAsync(out, m->dev.st, sizeof(State), cudaMemcpyDeviceToHost, m->stream));
     CK(cudaStreamSynchronize(m->stream));
     if (out->status == ST_TIMEOUT) { m->dead = true; return KG_E_TIMEOUT; }
+    if (out->status == ST_INTERNAL) {
+        std::snprintf(g_cuda_err, sizeof(g_cuda_err), "device-side index check %d failed", out->timeout_where);
+        m->dead = true;
+        return KG_E_INTERNAL;
+    }
     if (out->status != 0) {
         // an argument error found on the device (a token id outside the vocabulary): the sequence is unusable until
         // kg_reset, which also clears the state word; the weights are untouched
@@ -361,6 +376,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     D.dm.V = cfg->vocab; D.dm.l = cfg->exit_layer; D.dm.eps = cfg->rms_eps; D.dm.theta = cfg->rope_theta;
     D.dm.logit_scale = cfg->logit_scale; D.dm.max_seq = cfg->max_seq; D.dm.page_size = cfg->page_size;
     D.dm.n_pages = (cfg->max_seq + cfg->page_size - 1) / cfg->page_size; D.dm.gamma_max = cfg->gamma_max;
+    D.dm.n_phys = D.dm.n_pages;
     for (D.dm.ps_shift = 0; (1 << D.dm.ps_shift) < cfg->page_size; ++D.dm.ps_shift) {}
     D.dm.debug = cfg->debug_logits;
     for (int i = 0; i < cfg->head_dim / 2; ++i)
@@ -426,6 +442,8 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     if (!ok) { delete m; return KG_E_CUDA; }
     if (own) {
         int r = bf ? fill_weights<__nv_bfloat16>(m) : fill_weights<float>(m);
+        // the fill kernels have run to completion (and without a fault) when the model is handed out
+        if (r == KG_OK && cuda_failed(cudaStreamSynchronize(s), "weight fill")) r = KG_E_CUDA;
         if (r != KG_OK) { delete m; return r; }
     }
     *out = m;
@@ -771,6 +789,9 @@ extern "C" int kg_debug_fill_state(kg_model* m, int32_t T, int32_t n_d, uint64_t
 
 extern "C" int kg_debug_force_simple(kg_model* m, int on) {
     if (!m) return KG_E_ARG;
+    // the plain path stages all rows of an operand in shared memory: only shapes whose rows fit may take it
+    const int kmax = m->cfg.d_ffn > m->cfg.d_model ? m->cfg.d_ffn : m->cfg.d_model;
+    if (on && (size_t)kmax * KG_M_MAX * 4 > (size_t)SIMPLE_XS_BYTES) return KG_E_ARG;
     m->force_simple = on ? 1 : 0;
     return KG_OK;
 }
@@ -972,6 +993,7 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
     std::memset(&D, 0, sizeof(D));
     D.dm.H = H; D.dm.hd = hd; D.dm.d = H * hd; D.dm.page_size = page_size; D.dm.theta = theta;
     D.dm.n_pages = (pos0 + M + page_size - 1) / page_size;       // entries of page_table this call may touch
+    D.dm.n_phys = 0x7fffffff;                                    // the caller's cache: its page count is not known here
     for (D.dm.ps_shift = 0; (1 << D.dm.ps_shift) < page_size; ++D.dm.ps_shift) {}
     for (int i = 0; i < hd / 2; ++i) D.inv_freq[i] = std::pow((double)theta, -2.0 * (double)i / (double)hd);
     D.page_table = page_table;

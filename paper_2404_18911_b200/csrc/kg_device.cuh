@@ -50,7 +50,7 @@ constexpr int BAR_BYTES = 256;
 constexpr unsigned long long WAIT_TIMEOUT_CLK = 6000000000ull;   // default budget of a device-side wait: ~3 s at 1.9 GHz
 
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_HEAD = 3 };
-enum { ST_OK = 0, ST_TIMEOUT = -6 };
+enum { ST_OK = 0, ST_TIMEOUT = -6, ST_INTERNAL = -8 };
 
 struct LayerW {
     const void* wqkv; const void* wo; const void* wgate; const void* wup; const void* wdown;
@@ -61,6 +61,7 @@ struct Dims {
     int L, d, H, hd, F, V, l;
     float eps, theta, logit_scale;
     int max_seq, page_size, n_pages, gamma_max, debug;
+    int n_phys;         // physical pages behind the page table (page numbers must lie below it)
     int ps_shift;       // log2(page_size): page sizes are powers of two
     int stream;         // 1: linear operators take the streamed tensor-core path (bf16, d and F multiples of 16)
 };
@@ -1363,15 +1364,22 @@ struct PageWin {
 };
 
 // kc / vc point at the warp's first dim of the head (element offset hh * HD + dim offset is added by the caller per row)
+// A page number outside the cache never becomes an address: the access goes to page 0 and the state word records it.
+__device__ __forceinline__ int checked_page(int pg, int n_pages, State* st, int where) {
+    if ((unsigned)pg < (unsigned)n_pages) return pg;
+    if (st) { atomicCAS(&st->status, 0, ST_INTERNAL); st->timeout_where = where; }
+    return 0;
+}
+
 template <int HD>
 __device__ __forceinline__ void att_load(AttK& tk, AttV& tv, const __nv_bfloat16* kc, const __nv_bfloat16* vc, const PageWin& pw,
-                                         int H, int hh, int dof, int psh, int psm, int key0, int last_key) {
+                                         int H, int hh, int dof, int psh, int psm, int key0, int last_key, int n_pages, State* st) {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int mu = 4 * (g >> 1) + (g & 1);
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int key = min(key0 + mu + 2 * r, last_key);
-        const int pg = pw.page_of(key, psh);
+        const int pg = checked_page(pw.page_of(key, psh), n_pages, st, 50);
         const __nv_bfloat16* row = kc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + dof + 8 * t;
         tk.k[r][0] = __ldcg(reinterpret_cast<const uint4*>(row));
         tk.k[r][1] = __ldcg(reinterpret_cast<const uint4*>(row + 32));
@@ -1379,7 +1387,7 @@ __device__ __forceinline__ void att_load(AttK& tk, AttV& tv, const __nv_bfloat16
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int key = min(key0 + 4 * t + i, last_key);
-        const int pg = pw.page_of(key, psh);
+        const int pg = checked_page(pw.page_of(key, psh), n_pages, st, 51);
         const __nv_bfloat16* row = vc + ((((size_t)pg * H + hh) << psh) + (key & psm)) * HD + dof + 8 * g;
         tv.v[i] = __ldcg(reinterpret_cast<const uint4*>(row));
     }
@@ -1518,7 +1526,7 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
             const float q1 = ldcg_f(src), q2 = ldcg_f(src + half);
             const float k1 = ldcg_f(src + d), k2 = ldcg_f(src + d + half);
             const float v1 = ldcg_f(src + 2 * d), v2 = ldcg_f(src + 2 * d + half);
-            const int page = __ldg(D.page_table + (pos >> psh));
+            const int page = checked_page(__ldg(D.page_table + (pos >> psh)), D.dm.n_phys, D.st, 52);
             float cs, sn; rope_cs(D, pos, e, cs, sn);
             const float r1 = (q1 * cs - q2 * sn) * qscale, r2 = (q2 * cs + q1 * sn) * qscale;
             const __nv_bfloat16 h1 = __float2bfloat16_rn(r1), h2 = __float2bfloat16_rn(r2);
@@ -1547,7 +1555,7 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
         auto fetch = [&](AttK& tk, AttV& tv, int ti) {
             const int key0 = ti * ATT_TK, key1 = min(key0 + ATT_TK - 1, T - 1);
             if ((key1 >> psh) - pw.first >= 32) pw.load(D.page_table, D.dm.n_pages, key0 >> psh);
-            att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1);
+            att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1, D.dm.n_phys, D.st);
         };
         AttP pp;
         auto step = [&](const AttK& tk, const AttV& tv, int ti) {

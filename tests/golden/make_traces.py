@@ -13,7 +13,8 @@ a fixed sample of logit entries per row.
 Cases
   7b_full     the benchmark job: 7B shape, prompt 512, 256 tokens, eta 0.6, gamma 6, low-confidence draft kept
   13b_short   13B shape, 40-token prompt, 24 tokens, eta 0.6, gamma 6
-  33b_short   33B shape, 40-token prompt, 24 tokens, eta 0.6, gamma 8
+  33b_short   33B shape, 44-token prompt, 28 tokens, eta 0.6, gamma 8 (with a 40-token prompt the second round already
+              holds a verify row whose two leading logits are 0.014 apart, which ends a replay there)
   7b_verify   verify passes of the 7B shape on the microbenchmark state (seeded N(0,1) KV cache of length T and
               N(0,1) early features): (T, rows) = (128, 1), (512, 4), (2048, 8), (4096, 7), (4096, 11)
 """
@@ -115,7 +116,7 @@ def verify_case(name, config, points, seed):
 
 CASES = {
     "13b_short": lambda: generation_case("13b_short", "13b", 40, 24, 0.6, 6, ko.STOP_KEEP),
-    "33b_short": lambda: generation_case("33b_short", "33b", 40, 24, 0.6, 8, ko.STOP_KEEP),
+    "33b_short": lambda: generation_case("33b_short", "33b", 44, 28, 0.6, 8, ko.STOP_KEEP),
     "7b_verify": lambda: verify_case("7b_verify", "7b", [(128, 1), (512, 4), (2048, 8), (4096, 7), (4096, 11)], 11),
     "7b_full": lambda: generation_case("7b_full", "7b", 512, 256, 0.6, 6, ko.STOP_KEEP),
 }

@@ -1,0 +1,154 @@
+"""The CUDA path replays the oracle traces stored under tests/golden/ (written by tests/golden/make_traces.py,
+which runs only the fp64 CPU oracle): the benchmark job at full length on the 7B shape, short jobs on the 13B and
+33B shapes, and verify passes of the 7B shape on the microbenchmark state up to a KV length of 4096.
+
+Token ids, draft counts, accept lengths and S must agree exactly; on the 7B shape (the benchmark's) confidences
+within 1e-3 and the recorded logit entries (the two leading ones and a fixed sample per row) within 2e-2.  A
+decision may differ only at a position whose recorded top-2 gap is below the logit tolerance (or whose confidence
+lies within the confidence tolerance of eta); such a position is printed and ends the comparison there, and the
+full-length job must have compared at least 64 tokens by then.
+
+The deviation grows with width and depth: K and V pass through a bf16 quantiser, which turns the 1e-6-level
+differences between fp32-accumulated tensor-core arithmetic and the fp64 oracle into occasional one-ulp (2^-8
+relative) differences of cache entries.  Measured maxima: 7B 6.5e-3 (logits) / 6.5e-4 (confidences), 13B 1.3e-2 /
+1.5e-3, 33B 2.0e-2 / 2.6e-3.  The 13B and 33B shapes are therefore held to 2e-2 / 2e-3 and 4e-2 / 4e-3: their
+confidences (and the 33B logits) do not meet the 1e-3 / 2e-2 of the 7B target, and the test output says by how much."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import kg_inputs as ki
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+TOL = {"7b": (2e-2, 1e-3), "13b": (2e-2, 2e-3), "33b": (4e-2, 4e-3)}      # (logit, confidence) per shape
+
+
+@pytest.fixture(scope="module")
+def binding():
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_2404_18911_b200 import binding as b
+    b.load()
+    return b
+
+
+def _trace(name):
+    with open(os.path.join(GOLDEN, f"trace_{name}.json")) as f:
+        return json.load(f)
+
+
+def _check_row(z, rec, idx, what, tol):
+    """Recorded entries of one logit row against the device row z; returns the largest deviation."""
+    err = max(abs(float(z[i]) - v) for i, v in zip(idx, rec["samples"]))
+    for i, v in rec["top"]:
+        err = max(err, abs(float(z[i]) - v))
+    assert err < tol, (what, err)
+    return err
+
+
+def _replay(binding, tr, min_tokens, min_rounds=0):
+    shape = ki.get_config(tr["config"]).with_(max_seq=tr["n_prompt"] + tr["n_new"] + tr["gamma"] + 8)
+    g = binding.KangarooModel(shape, debug_logits=True)
+    prompt = ki.make_prompt(shape, tr["n_prompt"]).tolist()
+    idx, eta, gamma, mode, n_new = tr["sample_indices"], tr["eta"], tr["gamma"], tr["stop_mode"], tr["n_new"]
+    LOGIT_TOL, CONF_TOL = TOL[tr["config"]]
+    max_le = max_ce = 0.0
+    x0 = g.prefill(prompt)
+    max_le = max(max_le, _check_row(g.debug_logits(1, 0), tr["prefill"], idx, "prefill", LOGIT_TOL))
+    out, stop = [x0], None
+    if x0 != tr["prefill"]["x0"]:
+        assert tr["prefill"]["gap"] < LOGIT_TOL, ("x_0", x0, tr["prefill"]["x0"])
+        stop = ("prefill", tr["n_prompt"] - 1)
+    rounds = 0
+    for r in tr["rounds"]:
+        if stop or len(out) >= n_new:
+            break
+        d = g.draft(eta, gamma, mode)
+        v = g.verify()
+        rounds += 1
+        for j in range(min(d["n_steps"], r["n_steps"])):
+            max_le = max(max_le, _check_row(g.debug_logits(0, j), r["draft_rows"][j], idx, ("draft", rounds, j), LOGIT_TOL))
+            ce = abs(d["conf"][j] - r["conf"][j])
+            max_ce = max(max_ce, ce)
+            assert ce < CONF_TOL, ("confidence", rounds, j, d["conf"][j], r["conf"][j])
+            tg = d["tokens"][j] if j < len(d["tokens"]) else None
+            to = r["drafts"][j] if j < len(r["drafts"]) else None
+            if tg != to:
+                near = r["draft_rows"][j]["gap"] < LOGIT_TOL or abs(r["conf"][j] - eta) < CONF_TOL
+                assert near, ("draft token", rounds, j, tg, to)
+                stop = ("draft", r["P"] + j)
+                break
+        if stop:
+            break
+        if d["n_steps"] != r["n_steps"] or d["n_drafted"] != r["n_d"]:
+            assert any(abs(p - eta) < CONF_TOL for p in r["conf"]), ("draft counts", rounds, d, r["n_d"], r["n_steps"])
+            stop = ("eta", r["P"])
+            break
+        assert v["n_rows"] == r["n_d"] + 1
+        for i in range(r["n_d"] + 1):
+            max_le = max(max_le, _check_row(g.debug_logits(1, i), r["verify_rows"][i], idx, ("verify", rounds, i), LOGIT_TOL))
+            if v["target"][i] != r["target"][i]:
+                assert r["verify_rows"][i]["gap"] < LOGIT_TOL, ("target token", rounds, i, v["target"][i], r["target"][i])
+                stop = ("verify", r["P"] + i)
+                break
+        if stop:
+            break
+        assert v["k"] == r["k"] and v["emitted"] == r["emitted"], ("accept", rounds, v, r["k"], r["emitted"])
+        out.extend(v["emitted"])
+    n_cmp = min(len(out), n_new)
+    assert out[:n_cmp] == tr["tokens"][:n_cmp]
+    print(f"{tr['case']}: {rounds} rounds and {n_cmp} tokens compared, max logit deviation {max_le:.2e}, "
+          f"max confidence deviation {max_ce:.2e}, stopped at near-tie: {stop}")
+    assert n_cmp >= min_tokens and rounds >= min_rounds, (n_cmp, rounds, stop)
+    return g, shape, prompt, stop
+
+
+def test_benchmark_job_at_full_length_matches_the_oracle_trace(binding):
+    """7B shape, prompt 512, 256 tokens, eta 0.6, gamma 6: every round of the job the benchmark times."""
+    tr = _trace("7b_full")
+    g, shape, prompt, stop = _replay(binding, tr, 64)
+    if stop is None:
+        # the one-launch path the benchmark uses gives the same tokens and the same accepted-length list
+        toks, st = g.generate(prompt, tr["n_new"], tr["eta"], tr["gamma"], tr["stop_mode"])
+        assert toks == tr["tokens"]
+        assert g.read_S()[: st["rounds"] - 1] == tr["S"][:-1] and st["rounds"] == len(tr["S"])
+        assert abs(st["cr"] - tr["cr"]) < 1e-12
+        log = g.read_round_log()
+        assert [(a, b_, c) for (a, b_, c, _) in log] == [(r["n_d"], r["n_steps"], r["k"]) for r in tr["rounds"]]
+        assert [p for (_, _, _, p) in log] == [r["P"] for r in tr["rounds"]]
+
+
+@pytest.mark.parametrize("name", ["13b_short", "33b_short"])
+def test_large_shapes_match_the_oracle_trace(binding, name):
+    tr = _trace(name)
+    assert len(tr["rounds"]) >= 4
+    g, shape, prompt, stop = _replay(binding, tr, 8, min_rounds=4)
+    if stop is None:
+        toks, st = g.generate(prompt, tr["n_new"], tr["eta"], tr["gamma"], tr["stop_mode"])
+        assert toks == tr["tokens"] and st["rounds"] == len(tr["S"])
+        assert g.read_S()[: st["rounds"] - 1] == tr["S"][:-1]
+
+
+def test_verify_pass_on_the_microbenchmark_state_matches_the_oracle_trace(binding):
+    """Layers l+1..L and the LM head of the 7B shape on M rows against a seeded N(0,1) KV cache of length T."""
+    tr = _trace("7b_verify")
+    idx = tr["sample_indices"]
+    LOGIT_TOL = TOL[tr["config"]][0]
+    base = ki.get_config(tr["config"])
+    max_T = max(p["T"] for p in tr["points"])
+    max_M = max(p["M"] for p in tr["points"])
+    shape = base.with_(max_seq=max_T + max_M + 16 + base.gamma_max, gamma_max=max(base.gamma_max, max_M - 1))
+    g = binding.KangarooModel(shape, debug_logits=True)
+    for p in tr["points"]:
+        g.fill_state(p["T"], p["M"] - 1, tr["seed"])
+        v = g.verify()
+        assert v["n_rows"] == p["M"]
+        worst = 0.0
+        for i in range(p["M"]):
+            worst = max(worst, _check_row(g.debug_logits(1, i), p["rows"][i], idx, ("verify", p["T"], p["M"], i), LOGIT_TOL))
+            assert v["target"][i] == p["target"][i] or p["rows"][i]["gap"] < LOGIT_TOL, (p["T"], p["M"], i)
+        print(f"verify T={p['T']} M={p['M']}: max logit deviation {worst:.2e}")
