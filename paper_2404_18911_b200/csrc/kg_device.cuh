@@ -1478,7 +1478,8 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
     const int T = pos0 + M;
     const int ntiles_all = (T + ATT_TK - 1) / ATT_TK;
     const int R = (M + 7) >> 3;                       // row groups of 8
-    const int nw = NUNITS / R;                        // units that share the tiles of an item
+    const int nw = NUNITS / R;                        // units that share the tiles of an item (a power of two)
+    const int nw_sh = 31 - __clz(nw);
     // KV splits per head.  An item costs its units' tiles (one memory latency each) plus a fixed part, and a head
     // that is split pays for the merge of its partials through global memory (several dependent round trips, about
     // as long as three tiles): very short caches stay unsplit.
@@ -1489,7 +1490,7 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
 #pragma unroll
         for (int sc = 1; sc <= S_CAP; ++sc) {
             const int chunk_ = (ntiles_all + sc - 1) / sc;
-            const int tpw_ = (chunk_ + nw - 1) / nw;
+            const int tpw_ = (chunk_ + nw - 1) >> nw_sh;
             const float waves = ceilf((float)(H * sc) * inv_ctas - 1e-4f);
             const float cost = waves * (float)(tpw_ + 2 + (sc > 1 ? 3 : 0));
             if ((sc == 1 || chunk_ >= 2) && (best < 0.f || cost < best)) { best = cost; S = sc; }
@@ -1635,13 +1636,14 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
             cta_sync();
         }
         if (S > 1) {
-            __threadfence();
-            cta_sync();
+            // the partials of this CTA are ordered before the counter by the barrier above and the release of the
+            // atomic; the last arriver's acquire orders the counter before its reads of every split's partials
             if (tid == 0) {
-                const unsigned prev = atomicAdd(D.att_cnt + hh, 1u);
+                unsigned prev;
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(D.att_cnt + hh) : "memory");
                 const int last = (prev == (unsigned)(S - 1));
                 c.ctl->att_last = last;
-                if (last) { D.att_cnt[hh] = 0u; __threadfence(); }
+                if (last) D.att_cnt[hh] = 0u;
             }
             cta_sync();
             if (*(volatile int*)&c.ctl->att_last) {
