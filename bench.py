@@ -9,7 +9,10 @@ verify / accept rounds until n_gen tokens exist (Figure 2 of the paper), all on 
 already resident in HBM; `e2e` is the same job through kg_generate with pinned host buffers
 (prompt copied in, tokens copied out, every step).  The roofline object describes the decode
 launch (all rounds of a step run inside one persistent kernel launch): algorithmic bytes from the
-device's own per-round log divided by its CUDA-event duration.
+device's own per-round log divided by its CUDA-event duration.  Its `draft_step` and `verify_step`
+entries time single launches of one draft step (layers 1..l, adapter, LM head on one row) and of
+one verify pass (layers l+1..L and the LM head on M rows) against a KV cache of 512 tokens:
+>= 20 warm-up and >= 100 timed launches each, median with p10 / p90.
 
 With --gpus N > 1 (launched by torchrun) every rank runs an independent replica of the job: the
 batch-1 chain has no exchange step, so there is no collective on the data path.
@@ -205,11 +208,44 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32" if shape.d_model > 512 else "f64", "data": "synthetic",
-            "config": _config(shape, args, 1), "gpu_launches": 0,
+            "config": dict(_config(shape, args, 1), sample=sample), "gpu_launches": 0,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": _host_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
     return 0
+
+
+def _percentile(xs, q):
+    xs = sorted(xs)
+    return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
+
+
+def step_rooflines(model, shape, binding, traffic, torch, peak, T=512, Ms=(1, 4, 7), warm=20, reps=100):
+    """Single launches of one draft step and of one verify pass on the microbenchmark state (seeded N(0,1) KV cache of
+    length T, N(0,1) early features): algorithmic bytes / CUDA-event time of the launch, against the copy peak."""
+    def timed(prepare, launch, nbytes):
+        ms = []
+        for r in range(warm + reps):
+            prepare(r)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); launch(); e1.record()
+            torch.cuda.synchronize()
+            if r >= warm:
+                ms.append(e0.elapsed_time(e1))
+        med = statistics.median(ms)
+        return {"ms": med, "ms_p10": _percentile(ms, 0.1), "ms_p90": _percentile(ms, 0.9), "bytes": nbytes,
+                "achieved": nbytes / (med * 1e-3) / 1e9, "frac": nbytes / (med * 1e-3) / 1e9 / peak,
+                "frac_of_8TBs": nbytes / (med * 1e-3) / 1e9 / 8000.0, "launches": reps}
+    out = {"kv_len": T, "warmup": warm, "unit": "GB/s", "peak": peak}
+    # one draft step exactly: with eta > 1 in the stop mode that drops the low-confidence token the loop runs one
+    # shallow pass, one adapter + LM-head pass, and stops
+    out["draft_step"] = timed(lambda r: model.fill_state(T, -1, 100 + r),
+                              lambda: model.draft(2.0, 1, binding.STOP_DROP, sync=False), traffic.draft_step_bytes(shape, T))
+    out["verify_step"] = {}
+    for M in Ms:
+        out["verify_step"][f"M={M}"] = timed(lambda r, M=M: model.fill_state(T, M - 1, 200 + r),
+                                             lambda: model.verify(sync=False), traffic.verify_bytes(shape, T, M))
+    return out
 
 
 def _config(shape, args, world):
@@ -340,13 +376,19 @@ def run_kangaroo(args):
                          "frac_of_8TBs": achieved / 8000.0, "peak_source": peak_src,
                          "bytes_per_launch": dec_bytes, "ms_per_launch": dec_ms,
                          "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * dec_bytes),
-                         "traffic_source": "ncu dram bytes of a 4-layer launch of the same kernel, scaled by algorithmic bytes (x1.016)"},
+                         "traffic_source": None if NCU_TRAFFIC_RATIO is None else
+                         f"ncu dram bytes of a 4-layer launch of the same kernel, scaled by algorithmic bytes (x{NCU_TRAFFIC_RATIO})"},
             "breakdown": {"prefill_ms": statistics.mean(prefill_ms), "decode_ms": dec_ms,
                           "decode_only_tokens_per_s": (n_tok - 1) / (dec_ms * 1e-3),
                           "rounds": rounds, "cr": (n_tok - 1) / max(rounds, 1), "draft_steps": n_steps_total,
                           "drafted": drafted, "accepted": accepted,
                           "accept_rate": accepted / max(drafted, 1)},
         }
+        if not args.no_step_rooflines and not args.layers:
+            steps = step_rooflines(model, shape, binding, traffic, torch, peak)
+            line["roofline"]["draft_step"] = steps.pop("draft_step")
+            line["roofline"]["verify_step"] = steps.pop("verify_step")
+            line["roofline"]["step_timing"] = steps
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(args.workload)
         print(json.dumps(line), flush=True)
@@ -368,6 +410,7 @@ def main():
     ap.add_argument("--n-prompt", type=int, default=0, help="override the prompt length (profiling on a small case)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling on a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-step-rooflines", action="store_true", help="skip the single-launch draft-step / verify-step timings")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kangaroo" else args.warmup
     if args.impl == "reference":

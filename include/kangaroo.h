@@ -185,6 +185,10 @@ int kg_debug_force_simple(kg_model* m, int on);
 int kg_debug_force_simple_ops(int on);
 int kg_debug_set_wait_budget(kg_model* m, double milliseconds);
 int kg_debug_skip_barrier_arrival(kg_model* m, int cta);
+/* kg_debug_set_prefill_mode: 0 (default): prompts of 32 tokens and more take the tensor-core prompt pass when the
+ *   model is bf16 with head_dim 64 / 128 and d, F multiples of 128; 1: every prompt takes the 16-row chunked pass of
+ *   the decode kernels (the two are compared with each other and with the oracle in the tests). */
+int kg_debug_set_prefill_mode(kg_model* m, int mode);
 
 /* ---- single operators on caller buffers (unit tests and microbenchmarks) ------------------------
  * All pointers are device pointers, 16-byte aligned (int32 arrays: 4-byte), else KG_E_ARG; `scratch_dev` must hold

@@ -25,6 +25,7 @@ EXPORTS = [
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
     "kg_op_lm_head", "kg_op_lm_head_noalloc", "kg_op_attention", "kg_strerror",
     "kg_last_cuda_error", "kg_debug_force_simple", "kg_debug_force_simple_ops", "kg_debug_set_wait_budget", "kg_debug_skip_barrier_arrival",
+    "kg_debug_set_prefill_mode",
 ]
 
 
@@ -122,6 +123,7 @@ def load():
     lib.kg_debug_force_simple_ops.argtypes = [C.c_int]
     lib.kg_debug_set_wait_budget.argtypes = [vp, C.c_double]
     lib.kg_debug_skip_barrier_arrival.argtypes = [vp, C.c_int]
+    lib.kg_debug_set_prefill_mode.argtypes = [vp, C.c_int]
     _lib = lib
     return lib
 
@@ -327,6 +329,9 @@ class KangarooModel:
 
     def set_wait_budget(self, milliseconds):
         _check(self.lib.kg_debug_set_wait_budget(self.h, float(milliseconds)), "kg_debug_set_wait_budget")
+
+    def set_prefill_mode(self, mode):
+        _check(self.lib.kg_debug_set_prefill_mode(self.h, int(mode)), "kg_debug_set_prefill_mode")
 
     def skip_barrier_arrival(self, cta):
         _check(self.lib.kg_debug_skip_barrier_arrival(self.h, int(cta)), "kg_debug_skip_barrier_arrival")

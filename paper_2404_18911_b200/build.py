@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "csrc")
 _OUT = os.path.join(_HERE, "libkangaroo.so")
 _SOURCES = ["kg_api.cu"]
-_DEPS = ["kg_api.cu", "kg_engine.cuh", "kg_device.cuh", os.path.join("..", "..", "include", "kangaroo.h")]
+_DEPS = ["kg_api.cu", "kg_engine.cuh", "kg_device.cuh", "kg_prefill.cuh", os.path.join("..", "..", "include", "kangaroo.h")]
 
 
 def lib_path() -> str:

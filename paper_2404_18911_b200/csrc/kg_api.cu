@@ -10,6 +10,7 @@
 
 #include "../../include/kangaroo.h"
 #include "kg_engine.cuh"
+#include "kg_prefill.cuh"
 
 using namespace kg;
 
@@ -101,11 +102,19 @@ struct Layout {
     size_t off_hApk, off_hBpk, off_attnpk, off_actpk, off_featApk, off_featDpk, off_abufpk, off_ssqA, off_ssqB, off_ssqF, off_ssqAb;
     size_t off_layers, off_pt, off_kc, off_vc, off_h, off_feat, off_abuf, off_qkv, off_attn, off_act, off_po, off_ml,
         off_cnt, off_hp, off_dbgd, off_dbgv, off_out, off_S, off_rlog, off_prompt, off_st, off_bar;
+    // tensor-core prompt pass (0 bytes each when the shape cannot take it)
+    size_t off_pf_h, off_pf_h2, off_pf_qkv, off_pf_attn, off_pf_gate, off_pf_up, off_pf_hi, off_pf_lo, off_pf_err;
     size_t off_embed, off_head, off_gfinal;
     std::vector<size_t> off_w[5];     // wqkv, wo, wgate, wup, wdown
     std::vector<size_t> off_g[2];
     size_t total;
 };
+
+// The tensor-core prompt pass needs bf16 weights, a head_dim the tensor-core attention knows, and matrix sides that
+// are whole tiles: N a multiple of 128, K a multiple of 64.
+bool prefill_tc_shape(const kg_config* c) {
+    return c->dtype == KG_BF16 && (c->head_dim == 64 || c->head_dim == 128) && c->d_model % 128 == 0 && c->d_ffn % 128 == 0;
+}
 
 bool valid_config(const kg_config* c) {
     if (!c || c->struct_size != sizeof(kg_config)) return false;
@@ -118,6 +127,9 @@ bool valid_config(const kg_config* c) {
     if (c->page_size < 1 || (c->page_size & (c->page_size - 1)) || c->max_seq < 2) return false;       // pages hold a power of two of tokens
     if (c->n_heads > 256) return false;
     if (c->vocab > (1 << 20) || c->d_ffn > (1 << 20)) return false;      // rows x CTAs must fit 32 bits
+    // one launch may run max_seq tokens, each at most 5 (L + 1) + 8 grid barriers of at most 1024 CTAs: the arrival
+    // counter (31 bits beside the abort flag) must hold them all
+    if ((long long)c->max_seq * (5LL * (c->n_layers + 1) + 8) * 1024LL >= (1LL << 31)) return false;
     // the plain path stages all rows of an operand in shared memory
     const int kmax = c->d_ffn > c->d_model ? c->d_ffn : c->d_model;
     const bool plain_somewhere = c->dtype == KG_F32 || (c->d_model % 16) || (c->d_ffn % 16);
@@ -167,6 +179,12 @@ Layout make_layout(const kg_config* c, int own_weights, int nctas) {
     L.off_S = take(4 * (size_t)(c->max_seq + KG_M_MAX));
     L.off_rlog = take(16 * (size_t)(c->max_seq + KG_M_MAX));
     L.off_prompt = take(4 * (size_t)c->max_seq);
+    {
+        const size_t R = prefill_tc_shape(c) ? (size_t)PF_ROWS : 0, kmax = F > d ? F : d;
+        L.off_pf_h = take(4 * R * d); L.off_pf_h2 = take(4 * R * d); L.off_pf_qkv = take(4 * R * 3 * d);
+        L.off_pf_attn = take(4 * R * d); L.off_pf_gate = take(4 * R * F); L.off_pf_up = take(4 * R * F);
+        L.off_pf_hi = take(2 * R * kmax); L.off_pf_lo = take(2 * R * kmax); L.off_pf_err = take(R ? 256 : 0);
+    }
     for (int k = 0; k < 5; ++k) L.off_w[k].assign(nl + 1, 0);
     for (int k = 0; k < 2; ++k) L.off_g[k].assign(nl + 1, 0);
     L.off_embed = L.off_head = L.off_gfinal = 0;
@@ -225,6 +243,7 @@ struct kg_model {
     size_t smem;
     bool own_weights;
     bool prefilled, pending, ar_used, dead;
+    int prefill_mode;              // 0: tensor-core prompt pass when the shape and the prompt allow, 1: always the chunked pass
     unsigned long long wait_clk;   // budget of a device-side wait, in SM clocks
     int skip_arrival;              // test hook, consumed by the next launch
     cudaEvent_t ev0, ev1;          // timing of the decode loop in kg_generate, created on first use
@@ -361,7 +380,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     m->cfg = *cfg; m->lay = lay; m->arena = base; m->stream = (cudaStream_t)cuda_stream; m->nctas = nctas;
     m->own_weights = own != 0; m->prefilled = m->pending = m->ar_used = m->dead = false;
     m->gamma_pending = 0; m->P_upper = 0; m->force_simple = 0;
-    m->wait_clk = WAIT_TIMEOUT_CLK; m->skip_arrival = 0; m->ev0 = m->ev1 = nullptr;
+    m->wait_clk = WAIT_TIMEOUT_CLK; m->skip_arrival = 0; m->ev0 = m->ev1 = nullptr; m->prefill_mode = 0;
     m->smem = SMEM_TOTAL;
 
     const bool bf = cfg->dtype == KG_BF16;
@@ -382,7 +401,7 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     for (int i = 0; i < cfg->head_dim / 2; ++i)
         D.inv_freq[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
     auto P = [&](size_t off) { return base + off; };
-    D.st = (State*)P(lay.off_st); D.bar = (unsigned long long*)P(lay.off_bar);
+    D.st = (State*)P(lay.off_st); D.bar = (unsigned*)P(lay.off_bar);
     D.layers = (const LayerW*)P(lay.off_layers); D.page_table = (const int*)P(lay.off_pt);
     D.kcache = P(lay.off_kc); D.vcache = P(lay.off_vc);
     D.h = (float*)P(lay.off_h); D.feat = (float*)P(lay.off_feat); D.abuf = (float*)P(lay.off_abuf);
@@ -468,9 +487,19 @@ extern "C" int kg_reset(kg_model* m) {
     return KG_OK;
 }
 
+namespace {
+int prefill_tc(kg_model* m, int n);                 // the tensor-core prompt pass (end of this file)
+bool prefill_tc_ok(const kg_model* m, int n);
+}
+
 static int prefill_common(kg_model* m, int32_t n) {
-    Program pg{}; pg.kind = PROG_PREFILL; pg.n = n;
-    int r = launch(m, pg);
+    int r;
+    if (prefill_tc_ok(m, n)) {
+        r = prefill_tc(m, n);
+    } else {
+        Program pg{}; pg.kind = PROG_PREFILL; pg.n = n;
+        r = launch(m, pg);
+    }
     if (r != KG_OK) return r;
     m->prefilled = true; m->pending = false; m->P_upper = n;
     return KG_OK;
@@ -1010,5 +1039,148 @@ extern "C" int kg_op_attention(int32_t dtype, const float* qkv, int32_t M, int32
         op_attention_kernel<float><<<nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, a);
     }
     CK(cudaGetLastError());
+    return KG_OK;
+}
+
+// ------------------------------------------------------------------------------------ tensor-core prompt pass
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled of the driver, looked up through the runtime (the library does not link libcuda)
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows, K] read in boxes of 64 columns x 128 rows with the 128-byte swizzle.
+// base is 16-byte aligned and K * 2 a multiple of 16 (checked by the callers' shape test).
+bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {K, rows};
+    const cuuint64_t strides[1] = {K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)GM_BK, (cuuint32_t)GM_BM};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__global__ void __launch_bounds__(BLOCK_THREADS, 1) pf_attention_kernel(const __grid_constant__ Dev D, AttArgs a, int nrows) {
+    extern __shared__ __align__(128) char smem[];
+    Ctx& c = ctx_init(smem, nullptr, nullptr, false);
+    if (!c.producer) {
+        if (D.dm.hd == 128) attention_prefill<128>(D, a, c, nrows);
+        else attention_prefill<64>(D, a, c, nrows);
+    }
+}
+
+// x_0 from the per-CTA LM-head partials; the sequence state after a prompt of n tokens
+__global__ void pf_finish_kernel(const float4* part, int nctas, State* st, int* out_tokens, int n, const int* gemm_err) {
+    if (threadIdx.x == 0) {
+        int tok; float p;
+        head_final(part, nctas, 0, tok, p);
+        if (*gemm_err) { atomicCAS(&st->status, 0, ST_TIMEOUT); st->timeout_where = 60; }      // a wait inside a GEMM gave up
+        st->P = n; st->len_A = n; st->x0 = tok; st->pending = 0; st->total = 1; st->rounds = 0;
+        out_tokens[0] = tok;
+    }
+}
+
+bool prefill_tc_ok(const kg_model* m, int n) {
+    return m->prefill_mode == 0 && m->dev.dm.stream != 0 && prefill_tc_shape(&m->cfg) && n >= 2 * KG_M_MAX && encode_tiled_fn() != nullptr;
+}
+
+// C[rows, N] = (resid) + planes[rows, K] W[N, K]^T
+int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const float* resid) {
+    char* A = m->arena;
+    const int rows_pad = (rows + GM_BM - 1) / GM_BM * GM_BM;
+    CUtensorMap th, tl, tw;
+    if (!make_tmap(&th, A + m->lay.off_pf_hi, rows_pad, K) || !make_tmap(&tl, A + m->lay.off_pf_lo, rows_pad, K) || !make_tmap(&tw, W, N, K)) {
+        std::snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
+        return KG_E_CUDA;
+    }
+    GemmArgs g;
+    g.C = C; g.ldc = N; g.resid = resid; g.ldr = N; g.rows = rows; g.N = N; g.K = K; g.err = (int*)(A + m->lay.off_pf_err);
+    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, m->stream>>>(th, tl, tw, g);
+    CK(cudaGetLastError());
+    return KG_OK;
+}
+
+// The prompt in blocks of PF_ROWS rows, each block through all layers (its K / V are in the caches before the next
+// block attends to them), the adapter's K / V after layer l, the LM head on the last row.
+int prefill_tc(kg_model* m, int n) {
+    typedef __nv_bfloat16 WT;
+    const kg_config& c = m->cfg;
+    const Dev& D = m->dev;
+    cudaStream_t s = m->stream;
+    char* A = m->arena;
+    const int d = c.d_model, F = c.d_ffn, L = c.n_layers, H = c.n_heads;
+    float* h = (float*)(A + m->lay.off_pf_h); float* h2 = (float*)(A + m->lay.off_pf_h2);
+    float* qkv = (float*)(A + m->lay.off_pf_qkv); float* attn = (float*)(A + m->lay.off_pf_attn);
+    float* gate = (float*)(A + m->lay.off_pf_gate); float* up = (float*)(A + m->lay.off_pf_up);
+    WT* hi = (WT*)(A + m->lay.off_pf_hi); WT* lo = (WT*)(A + m->lay.off_pf_lo);
+    CK(cudaFuncSetAttribute((const void*)pf_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM));
+    CK(cudaFuncSetAttribute((const void*)pf_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL));
+    CK(cudaFuncSetAttribute((const void*)op_linear_kernel<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL));
+    CK(cudaMemsetAsync(A + m->lay.off_pf_err, 0, 4, s));
+    const size_t lstride = (size_t)D.dm.n_pages * H * c.page_size * c.head_dim;
+    int r = KG_OK;
+    for (int b0 = 0; b0 < n; b0 += PF_ROWS) {
+        const int rows = n - b0 < PF_ROWS ? n - b0 : PF_ROWS;
+        pf_embed_kernel<WT><<<rows, 256, 0, s>>>(D.prompt + b0, (const WT*)D.embed, c.vocab, d, h);
+        auto qkv_and_append = [&](const LayerW& lw, int li) -> int {
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h, d, d, lw.g1, c.rms_eps, hi, lo);
+            int rr = pf_gemm(m, lw.wqkv, 3 * d, d, rows, qkv, nullptr);
+            if (rr != KG_OK) return rr;
+            pf_rope_append_kernel<WT><<<dim3(rows, H), 64, 0, s>>>(D, qkv, b0, (WT*)D.kcache + (size_t)li * lstride, (WT*)D.vcache + (size_t)li * lstride);
+            return KG_OK;
+        };
+        for (int i = 0; i < L; ++i) {
+            const LayerW& lw = m->layers_host[i];
+            if ((r = qkv_and_append(lw, i)) != KG_OK) return r;
+            AttArgs at;
+            at.qkv = qkv; at.M = 0; at.pos0 = b0; at.kc = (WT*)D.kcache + (size_t)i * lstride; at.vc = (WT*)D.vcache + (size_t)i * lstride;
+            at.out = attn; at.opk = nullptr;
+            pf_attention_kernel<<<m->nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, at, rows);
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(attn, d, d, nullptr, 0.f, hi, lo);
+            if ((r = pf_gemm(m, lw.wo, d, d, rows, h2, h)) != KG_OK) return r;
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h2, d, d, lw.g2, c.rms_eps, hi, lo);
+            if ((r = pf_gemm(m, lw.wgate, F, d, rows, gate, nullptr)) != KG_OK) return r;
+            if ((r = pf_gemm(m, lw.wup, F, d, rows, up, nullptr)) != KG_OK) return r;
+            pf_swiglu_split_kernel<<<rows, 256, 0, s>>>(gate, up, F, hi, lo);
+            if ((r = pf_gemm(m, lw.wdown, d, F, rows, h, h2)) != KG_OK) return r;
+            if (i == c.exit_layer - 1 && (r = qkv_and_append(m->layers_host[L], L)) != KG_OK) return r;      // the adapter's K / V
+        }
+        CK(cudaGetLastError());
+    }
+    // LM head on the last prompt row (still in h): the decode path's fused head operator on one row
+    {
+        const int last = (n - 1) % PF_ROWS;
+        pack_rows_kernel<<<m->nctas, 256, 0, s>>>(h + (size_t)last * d, d, 1, d, D.g_final, D.hA_pk, d * 4, D.ssq_hA, m->nctas);
+        LinArgs a{};
+        a.W = D.head; a.N = c.vocab; a.K = d; a.M = 1; a.x = h + (size_t)last * d; a.ldx = d; a.gain = D.g_final; a.eps = c.rms_eps;
+        a.xpk = D.hA_pk; a.ldpk = d * 4; a.ssq_in = D.ssq_hA;
+        a.epi = EPI_HEAD; a.scale = c.logit_scale; a.head_part = D.head_part;
+        a.logits_dbg = c.debug_logits ? D.dbg_verify : nullptr; a.ld_dbg = c.vocab;
+        op_linear_kernel<WT><<<m->nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(a, 1);
+        pf_finish_kernel<<<1, 32, 0, s>>>(D.head_part, m->nctas, D.st, D.out_tokens, n, (const int*)(A + m->lay.off_pf_err));
+        CK(cudaGetLastError());
+    }
+    return KG_OK;
+}
+
+}  // namespace
+
+extern "C" int kg_debug_set_prefill_mode(kg_model* m, int mode) {
+    if (!m || (mode != 0 && mode != 1)) return KG_E_ARG;
+    m->prefill_mode = mode;
     return KG_OK;
 }

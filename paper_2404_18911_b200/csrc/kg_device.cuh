@@ -117,7 +117,7 @@ struct Dev {
     int* out_tokens; int* S; int* round_log;   // [max_seq], [max_seq], [max_seq][4]
     const int* prompt;             // device copy of the prompt
     State* st;
-    unsigned long long* bar;       // grid barrier arrival counter (zeroed before every launch)
+    unsigned* bar;                 // grid barrier arrival counter (zeroed before every launch)
     double inv_freq[HD_MAX / 2];   // theta^(-2i/hd)
 };
 
@@ -147,9 +147,9 @@ static_assert(sizeof(Ctrl) <= CTRL_BYTES - 16, "control block too large");
 // role's barriers; reading it never touches the per-thread stack.
 struct Ctx {
     int cta, nctas;
-    unsigned long long bar_target; // arrivals expected at the next grid barrier (thread 0 only)
+    unsigned bar_target;           // arrivals expected at the next grid barrier (thread 0 only)
     unsigned long long wait_clk;   // clocks after which a wait of this launch gives up
-    State* st; unsigned long long* bar;
+    State* st; unsigned* bar;
     int skip_arrival;              // test hook: 1 + index of the CTA that leaves out its first grid-barrier arrival (0: none)
     char* smem;
     Ctrl* ctl;
@@ -164,9 +164,9 @@ struct Ctx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
@@ -199,7 +199,7 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsign
 
 // The top bit of the grid barrier's arrival counter tells every CTA that some wait has given up: they learn it from
 // the word they poll anyway, without a second load.
-constexpr unsigned long long BAR_ABORT = 0x8000000000000000ull;
+constexpr unsigned BAR_ABORT = 0x80000000u;       // the host bounds a launch's arrivals below 2^31 (max_seq check)
 __device__ __forceinline__ void record_timeout(Ctx& c, int where) {
     *(volatile int*)&c.ctl->abort = 1;
     if (c.st) {
@@ -268,7 +268,7 @@ __device__ __forceinline__ bool arg_better(float za, int ia, float zb, int ib) {
 
 // ------------------------------------------------------------------------------------ CTA set-up
 // Called by every thread of the CTA at kernel start; returns the context of the thread's role.
-__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned long long* bar, bool grid,
+__device__ __forceinline__ Ctx& ctx_init(char* smem, State* st, unsigned* bar, bool grid,
                                          unsigned long long wait_clk = WAIT_TIMEOUT_CLK, int skip_arrival = 0) {
     static_assert(sizeof(Ctx) <= 128, "context slot too small");
     Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
@@ -299,18 +299,18 @@ __device__ __forceinline__ bool grid_sync(Ctx& c, int where) {
     if (!c.grid) { cta_sync(); return *(volatile int*)&c.ctl->abort == 0; }
     cta_sync();
     if (threadIdx.x == 0) {
-        // bar[0] counts arrivals (64 bits, monotonic over the launch): one release-add, then poll until every CTA has
-        // arrived or the abort bit appears
-        c.bar_target += (unsigned long long)c.nctas;
-        const unsigned long long gen = c.bar_target;
+        // bar[0] counts arrivals (monotonic over the launch, below 2^31: the host bounds max_seq accordingly): one
+        // release-add, then poll until every CTA has arrived or the abort bit appears
+        c.bar_target += (unsigned)c.nctas;
+        const unsigned gen = c.bar_target;
         if (c.skip_arrival == c.cta + 1) c.skip_arrival = 0;        // test hook: this arrival never happens
-        else asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(c.bar) : "memory");
+        else asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.bar) : "memory");
         int ok = 1;
         {
             const long long t0 = clock64();
             unsigned spins = 0;
             while (true) {
-                const unsigned long long v = ld_acquire_u64(c.bar);
+                const unsigned v = ld_acquire_u32(c.bar);
                 if (v & BAR_ABORT) { ok = 0; break; }
                 if (v >= gen) break;
                 if (((++spins) & 63u) == 0u) {
@@ -1464,8 +1464,11 @@ __device__ __forceinline__ void att_accumulate(const AttV& tv, AttAcc& ac, const
     }
 }
 
+// One work item of the tensor-core attention: head hh, split s of S (chunk_tiles tiles each) of the keys 0 .. pos0 + M - 1
+// for the rows of `a`.  append: this pass's K / V rows are rotated, rounded and written to the cache by the item whose
+// key range holds them (false: they are in the cache already).
 template <int HD>
-__device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& c) {
+__device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c, int hh, int s, int S, int chunk_tiles, bool append) {
     typedef __nv_bfloat16 WT;
     constexpr int NSPLIT = HD / ATT_DW;               // warps per unit: 1 (head_dim 64) or 2 (head_dim 128)
     constexpr int NUNITS = NWARPS / NSPLIT;
@@ -1479,6 +1482,167 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
     const int ntiles_all = (T + ATT_TK - 1) / ATT_TK;
     const int R = (M + 7) >> 3;                       // row groups of 8
     const int nw = NUNITS / R;                        // units that share the tiles of an item (a power of two)
+    const int tpw = (chunk_tiles + nw - 1) / nw;
+    const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;      // 1/sqrt(hd) and log2(e)
+    WT* kc = reinterpret_cast<WT*>(a.kc);
+    WT* vc = reinterpret_cast<WT*>(a.vc);
+    unsigned char* qs = reinterpret_cast<unsigned char*>(c.smem + WORK_OFF);
+    float* mb = reinterpret_cast<float*>(c.smem + WORK_OFF + AttSm<HD>::MB_OFF);
+    const int unit = warp / NSPLIT, hsel = warp % NSPLIT, dof = hsel * ATT_DW;
+    const int rg = unit % R, tlane = unit / R;
+    const int row0 = rg * 8;
+    const uint32_t qw = smem_u32(qs) + (uint32_t)(dof * 2);
+    // rows >= M of the row groups in use are zero in both planes
+    for (int idx = tid; idx < (8 * R - M) * half; idx += NTHREADS) {
+        const int i = M + idx / half, e = idx % half;
+        reinterpret_cast<unsigned*>(qs + (size_t)i * QS)[e] = 0u;
+        reinterpret_cast<unsigned*>(qs + (size_t)(M_MAX + i) * QS)[e] = 0u;
+    }
+    const int tb = s * chunk_tiles, te = min(ntiles_all, tb + chunk_tiles);
+    const int kb = tb * ATT_TK, ke = min(T, te * ATT_TK);
+    // this pass's rows: q rotated, scaled and split into the bf16 hi / lo planes; k rotated and, with v, rounded and
+    // appended to the cache when the row's position lies in my key range.  One cos / sin pair serves q and k, and
+    // all six loads of an element are issued before the first is used.
+    for (int idx = tid; idx < M * half; idx += NTHREADS) {
+        const int i = idx / half, e = idx % half, pos = pos0 + i;
+        const float* src = a.qkv + (size_t)i * 3 * d + hh * HD + e;
+        const float q1 = ldcg_f(src), q2 = ldcg_f(src + half);
+        const float k1 = ldcg_f(src + d), k2 = ldcg_f(src + d + half);
+        const float v1 = ldcg_f(src + 2 * d), v2 = ldcg_f(src + 2 * d + half);
+        const int page = checked_page(__ldg(D.page_table + (pos >> psh)), D.dm.n_phys, D.st, 52);
+        float cs, sn; rope_cs(D, pos, e, cs, sn);
+        const float r1 = (q1 * cs - q2 * sn) * qscale, r2 = (q2 * cs + q1 * sn) * qscale;
+        const __nv_bfloat16 h1 = __float2bfloat16_rn(r1), h2 = __float2bfloat16_rn(r2);
+        __nv_bfloat16* ph = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)i * QS);
+        __nv_bfloat16* pl = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)(M_MAX + i) * QS);
+        ph[e] = h1; ph[e + half] = h2;
+        pl[e] = __float2bfloat16_rn(r1 - __bfloat162float(h1)); pl[e + half] = __float2bfloat16_rn(r2 - __bfloat162float(h2));
+        if (append && pos >= kb && pos < ke) {
+            const size_t base = ((((size_t)page * H + hh) << psh) + (pos & psm)) * HD;
+            kc[base + e] = __float2bfloat16_rn(k1 * cs - k2 * sn);
+            kc[base + e + half] = __float2bfloat16_rn(k2 * cs + k1 * sn);
+            vc[base + e] = __float2bfloat16_rn(v1);
+            vc[base + e + half] = __float2bfloat16_rn(v2);
+        }
+    }
+    AttAcc ac;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
+    ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
+    // this unit's tiles: a contiguous run, so that one window of page-table entries serves many of them
+    int tile = tb + tlane * tpw;
+    const int tend = min(te, tile + tpw);
+    PageWin pw;
+    if (tile < tend) pw.load(D.page_table, D.dm.n_pages, (tile * ATT_TK) >> psh);
+    cta_sync();
+    auto fetch = [&](AttK& tk, AttV& tv, int ti) {
+        const int key0 = ti * ATT_TK, key1 = min(key0 + ATT_TK - 1, T - 1);
+        if ((key1 >> psh) - pw.first >= 32) pw.load(D.page_table, D.dm.n_pages, key0 >> psh);
+        att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1, D.dm.n_phys, D.st);
+    };
+    AttP pp;
+    auto step = [&](const AttK& tk, const AttV& tv, int ti) {
+        float sc[4];
+        att_scores<QS>(tk, sc, qw, row0);
+        if constexpr (NSPLIT == 2) {
+            // the pair's halves of the dot products meet in shared memory (two buffers, used alternately)
+            float4* xb = reinterpret_cast<float4*>(mb) + (size_t)((unit * 2 + (ti & 1)) * 2) * 32;
+            xb[hsel * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+            pair_sync(unit);
+            const float4 ot = xb[(hsel ^ 1) * 32 + lane];
+            sc[0] += ot.x; sc[1] += ot.y; sc[2] += ot.z; sc[3] += ot.w;
+        }
+        att_softmax(sc, ac, pp, row0, ti * ATT_TK, ke, pos0);
+        att_accumulate(tv, ac, pp);
+    };
+    // One register set for K and V (a second one would not fit: the register allocation is shared with the
+    // linear operators).  A tile therefore costs a memory latency; the split count above keeps the run of
+    // tiles per unit short, and the other units and CTAs keep the memory system busy meanwhile.
+    AttK k0;
+    AttV v0;
+    while (tile < tend) {
+        fetch(k0, v0, tile);
+        step(k0, v0, tile);
+        ++tile;
+    }
+    // the row sums: lanes that share rows add their shares in a fixed order
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 4);
+        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 8);
+        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 16);
+    }
+    if constexpr (NSPLIT == 2) cta_sync();          // the merge buffer lies over the pairs' exchange buffers
+    // merge the units of a row group through shared memory, four rows at a time
+    for (int rb = 0; rb * ATT_RB < M; ++rb) {
+        const int nr = min(ATT_RB, M - rb * ATT_RB);
+        if (rg == (rb >> 1) && (t >> 1) == (rb & 1)) {
+            const int rl = 2 * (t & 1);
+            float* r0 = mb + ((size_t)tlane * ATT_RB + rl) * ATT_MB_STRIDE;
+            float* r1 = r0 + ATT_MB_STRIDE;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int dd = dof + 8 * g + 2 * e;
+                *reinterpret_cast<float2*>(r0 + dd) = make_float2(ac.o[e][0], ac.o[e][2]);
+                *reinterpret_cast<float2*>(r1 + dd) = make_float2(ac.o[e][1], ac.o[e][3]);
+            }
+            if (g == 0 && hsel == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
+        }
+        cta_sync();
+        for (int idx = tid; idx < nr * HD; idx += NTHREADS) {
+            const int r = idx / HD, e = idx % HD, i = rb * ATT_RB + r;
+            float mx = -INFINITY;
+            for (int w = 0; w < nw; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
+            float den = 0.f, num = 0.f;
+            for (int w = 0; w < nw; ++w) {
+                const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
+                const float mw = row[HD_MAX];
+                if (mw != -INFINITY) {
+                    const float wgt = ex2f(mw - mx);
+                    den += row[HD_MAX + 1] * wgt;
+                    num += row[e] * wgt;
+                }
+            }
+            if (S == 1) {
+                const float ov = num / den;
+                a.out[(size_t)i * d + hh * HD + e] = ov;
+                if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * HD + e, ov);
+            } else {
+                D.att_po[(((size_t)i * H + hh) * S_CAP + s) * HD + e] = num;
+                if (e == 0) {
+                    D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 0] = mx;
+                    D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 1] = den;
+                }
+            }
+        }
+        cta_sync();
+    }
+    if (S > 1) {
+        // the partials of this CTA are ordered before the counter by the barrier above and the release of the
+        // atomic; the last arriver's acquire orders the counter before its reads of every split's partials
+        if (tid == 0) {
+            unsigned prev;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(D.att_cnt + hh) : "memory");
+            const int last = (prev == (unsigned)(S - 1));
+            c.ctl->att_last = last;
+            if (last) D.att_cnt[hh] = 0u;
+        }
+        cta_sync();
+        if (*(volatile int*)&c.ctl->att_last) {
+            if (S <= 4) att_merge_splits<4, 4>(D, a, hh, S, M);
+            else if (S <= 8) att_merge_splits<8, 2>(D, a, hh, S, M);
+            else att_merge_splits<S_CAP, 1>(D, a, hh, S, M);
+        }
+        cta_sync();
+    }
+}
+
+template <int HD>
+__device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& c) {
+    constexpr int NUNITS = NWARPS / (HD / ATT_DW);
+    const int H = D.dm.H;
+    const int ntiles_all = (a.pos0 + a.M + ATT_TK - 1) / ATT_TK;
+    const int nw = NUNITS / ((a.M + 7) >> 3);
     const int nw_sh = 31 - __clz(nw);
     // KV splits per head.  An item costs its units' tiles (one memory latency each) plus a fixed part, and a head
     // that is split pays for the merge of its partials through global memory (several dependent round trips, about
@@ -1497,162 +1661,24 @@ __device__ __noinline__ void attention_mma(const Dev& D, const AttArgs& a, Ctx& 
         }
     }
     const int chunk_tiles = (ntiles_all + S - 1) / S;
-    const int tpw = (chunk_tiles + nw - 1) / nw;
-    const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;      // 1/sqrt(hd) and log2(e)
-    WT* kc = reinterpret_cast<WT*>(a.kc);
-    WT* vc = reinterpret_cast<WT*>(a.vc);
-    unsigned char* qs = reinterpret_cast<unsigned char*>(c.smem + WORK_OFF);
-    float* mb = reinterpret_cast<float*>(c.smem + WORK_OFF + AttSm<HD>::MB_OFF);
-    const int unit = warp / NSPLIT, hsel = warp % NSPLIT, dof = hsel * ATT_DW;
-    const int rg = unit % R, tlane = unit / R;
-    const int row0 = rg * 8;
-    const uint32_t qw = smem_u32(qs) + (uint32_t)(dof * 2);
-    // rows >= M of the row groups in use are zero in both planes
-    for (int idx = tid; idx < (8 * R - M) * half; idx += NTHREADS) {
-        const int i = M + idx / half, e = idx % half;
-        reinterpret_cast<unsigned*>(qs + (size_t)i * QS)[e] = 0u;
-        reinterpret_cast<unsigned*>(qs + (size_t)(M_MAX + i) * QS)[e] = 0u;
-    }
+    for (int item = c.cta; item < H * S; item += c.nctas) att_item<HD>(D, a, c, item / S, item % S, S, chunk_tiles, true);
+}
 
-    for (int item = c.cta; item < H * S; item += c.nctas) {
-        const int hh = item / S, s = item % S;
-        const int tb = s * chunk_tiles, te = min(ntiles_all, tb + chunk_tiles);
-        const int kb = tb * ATT_TK, ke = min(T, te * ATT_TK);
-        // this pass's rows: q rotated, scaled and split into the bf16 hi / lo planes; k rotated and, with v, rounded and
-        // appended to the cache when the row's position lies in my key range.  One cos / sin pair serves q and k, and
-        // all six loads of an element are issued before the first is used.
-        for (int idx = tid; idx < M * half; idx += NTHREADS) {
-            const int i = idx / half, e = idx % half, pos = pos0 + i;
-            const float* src = a.qkv + (size_t)i * 3 * d + hh * HD + e;
-            const float q1 = ldcg_f(src), q2 = ldcg_f(src + half);
-            const float k1 = ldcg_f(src + d), k2 = ldcg_f(src + d + half);
-            const float v1 = ldcg_f(src + 2 * d), v2 = ldcg_f(src + 2 * d + half);
-            const int page = checked_page(__ldg(D.page_table + (pos >> psh)), D.dm.n_phys, D.st, 52);
-            float cs, sn; rope_cs(D, pos, e, cs, sn);
-            const float r1 = (q1 * cs - q2 * sn) * qscale, r2 = (q2 * cs + q1 * sn) * qscale;
-            const __nv_bfloat16 h1 = __float2bfloat16_rn(r1), h2 = __float2bfloat16_rn(r2);
-            __nv_bfloat16* ph = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)i * QS);
-            __nv_bfloat16* pl = reinterpret_cast<__nv_bfloat16*>(qs + (size_t)(M_MAX + i) * QS);
-            ph[e] = h1; ph[e + half] = h2;
-            pl[e] = __float2bfloat16_rn(r1 - __bfloat162float(h1)); pl[e + half] = __float2bfloat16_rn(r2 - __bfloat162float(h2));
-            if (pos >= kb && pos < ke) {
-                const size_t base = ((((size_t)page * H + hh) << psh) + (pos & psm)) * HD;
-                kc[base + e] = __float2bfloat16_rn(k1 * cs - k2 * sn);
-                kc[base + e + half] = __float2bfloat16_rn(k2 * cs + k1 * sn);
-                vc[base + e] = __float2bfloat16_rn(v1);
-                vc[base + e + half] = __float2bfloat16_rn(v2);
-            }
-        }
-        AttAcc ac;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
-        ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
-        // this unit's tiles: a contiguous run, so that one window of page-table entries serves many of them
-        int tile = tb + tlane * tpw;
-        const int tend = min(te, tile + tpw);
-        PageWin pw;
-        if (tile < tend) pw.load(D.page_table, D.dm.n_pages, (tile * ATT_TK) >> psh);
-        cta_sync();
-        auto fetch = [&](AttK& tk, AttV& tv, int ti) {
-            const int key0 = ti * ATT_TK, key1 = min(key0 + ATT_TK - 1, T - 1);
-            if ((key1 >> psh) - pw.first >= 32) pw.load(D.page_table, D.dm.n_pages, key0 >> psh);
-            att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1, D.dm.n_phys, D.st);
-        };
-        AttP pp;
-        auto step = [&](const AttK& tk, const AttV& tv, int ti) {
-            float sc[4];
-            att_scores<QS>(tk, sc, qw, row0);
-            if constexpr (NSPLIT == 2) {
-                // the pair's halves of the dot products meet in shared memory (two buffers, used alternately)
-                float4* xb = reinterpret_cast<float4*>(mb) + (size_t)((unit * 2 + (ti & 1)) * 2) * 32;
-                xb[hsel * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
-                pair_sync(unit);
-                const float4 ot = xb[(hsel ^ 1) * 32 + lane];
-                sc[0] += ot.x; sc[1] += ot.y; sc[2] += ot.z; sc[3] += ot.w;
-            }
-            att_softmax(sc, ac, pp, row0, ti * ATT_TK, ke, pos0);
-            att_accumulate(tv, ac, pp);
-        };
-        // One register set for K and V (a second one would not fit: the register allocation is shared with the
-        // linear operators).  A tile therefore costs a memory latency; the split count above keeps the run of
-        // tiles per unit short, and the other units and CTAs keep the memory system busy meanwhile.
-        AttK k0;
-        AttV v0;
-        while (tile < tend) {
-            fetch(k0, v0, tile);
-            step(k0, v0, tile);
-            ++tile;
-        }
-        // the row sums: lanes that share rows add their shares in a fixed order
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 4);
-            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 8);
-            ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 16);
-        }
-        if constexpr (NSPLIT == 2) cta_sync();          // the merge buffer lies over the pairs' exchange buffers
-        // merge the units of a row group through shared memory, four rows at a time
-        for (int rb = 0; rb * ATT_RB < M; ++rb) {
-            const int nr = min(ATT_RB, M - rb * ATT_RB);
-            if (rg == (rb >> 1) && (t >> 1) == (rb & 1)) {
-                const int rl = 2 * (t & 1);
-                float* r0 = mb + ((size_t)tlane * ATT_RB + rl) * ATT_MB_STRIDE;
-                float* r1 = r0 + ATT_MB_STRIDE;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int dd = dof + 8 * g + 2 * e;
-                    *reinterpret_cast<float2*>(r0 + dd) = make_float2(ac.o[e][0], ac.o[e][2]);
-                    *reinterpret_cast<float2*>(r1 + dd) = make_float2(ac.o[e][1], ac.o[e][3]);
-                }
-                if (g == 0 && hsel == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
-            }
-            cta_sync();
-            for (int idx = tid; idx < nr * HD; idx += NTHREADS) {
-                const int r = idx / HD, e = idx % HD, i = rb * ATT_RB + r;
-                float mx = -INFINITY;
-                for (int w = 0; w < nw; ++w) mx = fmaxf(mx, mb[((size_t)w * ATT_RB + r) * ATT_MB_STRIDE + HD_MAX]);
-                float den = 0.f, num = 0.f;
-                for (int w = 0; w < nw; ++w) {
-                    const float* row = mb + ((size_t)w * ATT_RB + r) * ATT_MB_STRIDE;
-                    const float mw = row[HD_MAX];
-                    if (mw != -INFINITY) {
-                        const float wgt = ex2f(mw - mx);
-                        den += row[HD_MAX + 1] * wgt;
-                        num += row[e] * wgt;
-                    }
-                }
-                if (S == 1) {
-                    const float ov = num / den;
-                    a.out[(size_t)i * d + hh * HD + e] = ov;
-                    if (a.opk) pk_store(a.opk + (size_t)i * d * 4, hh * HD + e, ov);
-                } else {
-                    D.att_po[(((size_t)i * H + hh) * S_CAP + s) * HD + e] = num;
-                    if (e == 0) {
-                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 0] = mx;
-                        D.att_ml[(((size_t)i * H + hh) * S_CAP + s) * 2 + 1] = den;
-                    }
-                }
-            }
-            cta_sync();
-        }
-        if (S > 1) {
-            // the partials of this CTA are ordered before the counter by the barrier above and the release of the
-            // atomic; the last arriver's acquire orders the counter before its reads of every split's partials
-            if (tid == 0) {
-                unsigned prev;
-                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(D.att_cnt + hh) : "memory");
-                const int last = (prev == (unsigned)(S - 1));
-                c.ctl->att_last = last;
-                if (last) D.att_cnt[hh] = 0u;
-            }
-            cta_sync();
-            if (*(volatile int*)&c.ctl->att_last) {
-                if (S <= 4) att_merge_splits<4, 4>(D, a, hh, S, M);
-                else if (S <= 8) att_merge_splits<8, 2>(D, a, hh, S, M);
-                else att_merge_splits<S_CAP, 1>(D, a, hh, S, M);
-            }
-            cta_sync();
-        }
+// The prompt pass: `nrows` rows at positions a.pos0.. whose K / V are in the cache already; an item is a block of 16
+// rows of one head against all keys it may see (no splits: there are plenty of items).
+template <int HD>
+__device__ __noinline__ void attention_prefill(const Dev& D, const AttArgs& a, Ctx& c, int nrows) {
+    const int H = D.dm.H, d = D.dm.d;
+    const int nblk = (nrows + M_MAX - 1) / M_MAX;
+    for (int item = c.cta; item < nblk * H; item += c.nctas) {
+        const int rb = item / H, hh = item % H;
+        AttArgs b = a;
+        b.qkv = a.qkv + (size_t)rb * M_MAX * 3 * d;
+        b.out = a.out + (size_t)rb * M_MAX * d;
+        b.opk = nullptr;
+        b.M = min(M_MAX, nrows - rb * M_MAX);
+        b.pos0 = a.pos0 + rb * M_MAX;
+        att_item<HD>(D, b, c, hh, 0, 1, (b.pos0 + b.M + ATT_TK - 1) / ATT_TK, false);
     }
 }
 static_assert(AttSm<HD_MAX>::MB_OFF + NWARPS * ATT_RB * ATT_MB_STRIDE * 4 <= WORK_BYTES, "tensor-core attention buffers do not fit in the work area");

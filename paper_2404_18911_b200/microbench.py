@@ -1,13 +1,14 @@
 """Step and operator microbenchmarks of the decode path (the verify-step / draft-step evaluation shapes).
 
     python -m paper_2404_18911_b200.microbench [--workload 7b] [--what steps|ops|all] [--T 128,512,2048,4096]
-                                               [--M 1,2,4,7,8] [--reps 10]
+                                               [--M 1,2,3,4,5,6,7,8,9,10,11,16] [--warmup 20] [--reps 100]
 
 steps: the verify pass (layers l+1..L + head on M rows) against a seeded N(0,1) KV cache of length T,
        the draft loop with eta = 0 (gamma full draft steps + one shallow pass), and plain AR steps;
 ops:   each linear operator of a layer and the LM head as a single launch, rotating over enough
        weight copies that no launch finds its weights in L2.
-Prints one JSON object per point: time, algorithmic bytes, achieved GB/s.
+Prints one JSON object per point: median time with p10 / p90 over the timed launches (after the warm-up launches),
+algorithmic bytes, achieved GB/s.
 """
 from __future__ import annotations
 
@@ -21,6 +22,11 @@ def _events(torch):
     return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
 
+def _pct(xs, q):
+    xs = sorted(xs)
+    return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
+
+
 def bench_steps(args, shape, torch, binding, traffic):
     Ts = [int(t) for t in args.T.split(",")]
     Ms = [int(m) for m in args.M.split(",")]
@@ -31,36 +37,53 @@ def bench_steps(args, shape, torch, binding, traffic):
     for T in Ts:
         for M in Ms:
             ms = []
-            for r in range(args.reps + 2):
+            for r in range(args.reps + args.warmup):
                 model.fill_state(T, M - 1, 7 + r)
                 e0, e1 = _events(torch)
                 e0.record()
                 model.verify(sync=False)
                 e1.record()
                 torch.cuda.synchronize()
-                if r >= 2:
+                if r >= args.warmup:
                     ms.append(e0.elapsed_time(e1))
             b = traffic.verify_bytes(shape, T, M)
             t = statistics.median(ms)
-            out.append({"point": "verify", "T": T, "M": M, "ms": t, "ms_min": min(ms), "bytes": b, "GBps": b / t / 1e6})
+            out.append({"point": "verify", "T": T, "M": M, "ms": t, "ms_p10": _pct(ms, 0.1), "ms_p90": _pct(ms, 0.9), "bytes": b,
+                        "GBps": b / t / 1e6, "launches": len(ms)})
             print(json.dumps(out[-1]), flush=True)
         # draft loop, eta = 0: gamma adapter+head steps and gamma+1 shallow passes
         g = min(shape.gamma_max, 10)
         ms = []
-        for r in range(args.reps + 2):
+        for r in range(args.reps + args.warmup):
             model.fill_state(T, -1, 7 + r)
             e0, e1 = _events(torch)
             e0.record()
             model.draft(0.0, g, binding.STOP_KEEP, sync=False)
             e1.record()
             torch.cuda.synchronize()
-            if r >= 2:
+            if r >= args.warmup:
                 ms.append(e0.elapsed_time(e1))
         b = sum(traffic.shallow_pass_bytes(shape, T + j) for j in range(g + 1)) + \
             sum(traffic.adapter_head_bytes(shape, T + j, 1) for j in range(g))
         t = statistics.median(ms)
         out.append({"point": "draft_loop", "T": T, "gamma": g, "ms": t, "ms_per_draft_step": t / (g + 0.5), "bytes": b,
                     "GBps": b / t / 1e6})
+        print(json.dumps(out[-1]), flush=True)
+        # one draft step exactly (one shallow pass, one adapter + LM-head pass): eta > 1, low-confidence token dropped
+        ms = []
+        for r in range(args.reps + args.warmup):
+            model.fill_state(T, -1, 7 + r)
+            e0, e1 = _events(torch)
+            e0.record()
+            model.draft(2.0, 1, binding.STOP_DROP, sync=False)
+            e1.record()
+            torch.cuda.synchronize()
+            if r >= args.warmup:
+                ms.append(e0.elapsed_time(e1))
+        b = traffic.draft_step_bytes(shape, T)
+        t = statistics.median(ms)
+        out.append({"point": "draft_step", "T": T, "ms": t, "ms_p10": _pct(ms, 0.1), "ms_p90": _pct(ms, 0.9), "bytes": b,
+                    "GBps": b / t / 1e6, "launches": len(ms)})
         print(json.dumps(out[-1]), flush=True)
         # plain AR
         n = 8
@@ -149,8 +172,9 @@ def main():
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--what", default="steps", choices=["steps", "ops", "sweep", "all"])
     ap.add_argument("--T", default="128,512,2048,4096")
-    ap.add_argument("--M", default="1,2,4,7,8")
-    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--M", default="1,2,3,4,5,6,7,8,9,10,11,16")
+    ap.add_argument("--reps", type=int, default=100, help="timed launches per point")
+    ap.add_argument("--warmup", type=int, default=20, help="untimed launches per point")
     args = ap.parse_args()
     build_library()
     binding.load()
