@@ -226,6 +226,13 @@ int kg_op_lm_head_noalloc(int32_t dtype, const void* W_head_dev, int32_t V, int3
                           const float* gain_dev, float eps, float logit_scale,
                           int32_t* tok_dev, float* p_dev, float* logits_dev, void* cuda_stream);
 
+/* The GEMM of the tensor-core prompt pass (the state Figure 2 starts from is built with it): out[M, N] = (resid ? resid : 0)
+ * + x W^T for bf16 W [N, K] and fp32 x [M, K], any M >= 1; x is split into two bf16 planes (x = hi + lo) and both are
+ * multiplied with W on the tensor cores into fp32.  N a multiple of 128, K a multiple of 64 (else KG_E_ARG);
+ * ceil(M / 128) * 128 * K <= 2097152 elements so that the planes fit in `scratch_dev` (else KG_E_LIMIT). */
+int kg_op_gemm(const void* W_dev, int32_t N, int32_t K, const float* x_dev, int32_t M, const float* resid_dev, float* out_dev,
+               void* scratch_dev, void* cuda_stream);
+
 /* Causal attention of M new rows at positions pos0.. over a paged KV cache (RoPE fused): takes the
  * raw q,k,v rows qkv[M, 3d], rotates q and k, appends k and v to the cache pages, and returns
  * out[M, d] = concat_heads softmax(q K^T / sqrt(hd)) V.  Cache layout: [page][head][slot][hd]. */

@@ -25,7 +25,7 @@ EXPORTS = [
     "kg_debug_logits", "kg_read_weight", "kg_debug_fill_state", "kg_op_scratch_bytes", "kg_op_linear",
     "kg_op_lm_head", "kg_op_lm_head_noalloc", "kg_op_attention", "kg_strerror",
     "kg_last_cuda_error", "kg_debug_force_simple", "kg_debug_force_simple_ops", "kg_debug_set_wait_budget", "kg_debug_skip_barrier_arrival",
-    "kg_debug_set_prefill_mode",
+    "kg_debug_set_prefill_mode", "kg_op_gemm",
 ]
 
 
@@ -115,6 +115,7 @@ def load():
     lib.kg_op_lm_head.argtypes = [i32, vp, i32, i32, vp, i32, vp, f32, f32, vp, vp, vp, vp, vp]
     lib.kg_op_lm_head_noalloc.argtypes = [i32, vp, i32, i32, vp, i32, vp, f32, f32, vp, vp, vp, vp]
     lib.kg_op_attention.argtypes = [i32, vp, i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, vp, vp]
+    lib.kg_op_gemm.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp]
     lib.kg_strerror.restype = C.c_char_p
     lib.kg_strerror.argtypes = [C.c_int]
     lib.kg_last_cuda_error.restype = C.c_char_p
@@ -361,6 +362,17 @@ def op_linear(W, x, gain=None, eps=1e-6, resid=None, W2=None, scratch=None):
     scratch = op_scratch(torch, x.device) if scratch is None else scratch
     _check(lib.kg_op_linear(dt, W.data_ptr(), _ptr(W2), N, K, x.data_ptr(), M, _ptr(gain), eps, _ptr(resid),
                             int(W2 is not None), out.data_ptr(), scratch.data_ptr(), _stream(torch)), "kg_op_linear")
+    return out
+
+
+def op_gemm(W, x, resid=None, scratch=None):
+    import torch
+    lib = load()
+    N, K = W.shape
+    M = x.shape[0]
+    out = torch.empty(M, N, dtype=torch.float32, device=x.device)
+    scratch = op_scratch(torch, x.device) if scratch is None else scratch
+    _check(lib.kg_op_gemm(W.data_ptr(), N, K, x.data_ptr(), M, _ptr(resid), out.data_ptr(), scratch.data_ptr(), _stream(torch)), "kg_op_gemm")
     return out
 
 

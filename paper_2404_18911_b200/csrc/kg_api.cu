@@ -183,7 +183,7 @@ Layout make_layout(const kg_config* c, int own_weights, int nctas) {
         const size_t R = prefill_tc_shape(c) ? (size_t)PF_ROWS : 0, kmax = F > d ? F : d;
         L.off_pf_h = take(4 * R * d); L.off_pf_h2 = take(4 * R * d); L.off_pf_qkv = take(4 * R * 3 * d);
         L.off_pf_attn = take(4 * R * d); L.off_pf_gate = take(4 * R * F); L.off_pf_up = take(4 * R * F);
-        L.off_pf_hi = take(2 * R * kmax); L.off_pf_lo = take(2 * R * kmax); L.off_pf_err = take(R ? 256 : 0);
+        L.off_pf_hi = take(2 * R * kmax); L.off_pf_lo = take(2 * R * kmax); L.off_pf_err = take(R ? 64 + 4 * R : 0);      // error word, then 1/rms per row
     }
     for (int k = 0; k < 5; ++k) L.off_w[k].assign(nl + 1, 0);
     for (int k = 0; k < 2; ++k) L.off_g[k].assign(nl + 1, 0);
@@ -273,7 +273,7 @@ extern "C" const char* kg_strerror(int s) {
         case KG_E_SEQ_FULL: return "sequence would exceed max_seq";
         case KG_E_CUDA: return "CUDA runtime error";
         case KG_E_TIMEOUT: return "device-side wait timed out";
-        case KG_E_LIMIT: return "size beyond the capacity of the library's static scratch";
+        case KG_E_LIMIT: return "size beyond the capacity of the library's static scratch (or of the operator scratch)";
         case KG_E_INTERNAL: return "a device-side index check failed (the access was skipped)";
         default: return "unknown status";
     }
@@ -1099,7 +1099,7 @@ bool prefill_tc_ok(const kg_model* m, int n) {
 }
 
 // C[rows, N] = (resid) + planes[rows, K] W[N, K]^T
-int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const float* resid) {
+int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const float* resid, const float* rowscale) {
     char* A = m->arena;
     const int rows_pad = (rows + GM_BM - 1) / GM_BM * GM_BM;
     CUtensorMap th, tl, tw;
@@ -1108,7 +1108,7 @@ int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const 
         return KG_E_CUDA;
     }
     GemmArgs g;
-    g.C = C; g.ldc = N; g.resid = resid; g.ldr = N; g.rows = rows; g.N = N; g.K = K; g.err = (int*)(A + m->lay.off_pf_err);
+    g.C = C; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = rowscale; g.rows = rows; g.N = N; g.K = K; g.err = (int*)(A + m->lay.off_pf_err);
     pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, m->stream>>>(th, tl, tw, g);
     CK(cudaGetLastError());
     return KG_OK;
@@ -1127,6 +1127,7 @@ int prefill_tc(kg_model* m, int n) {
     float* qkv = (float*)(A + m->lay.off_pf_qkv); float* attn = (float*)(A + m->lay.off_pf_attn);
     float* gate = (float*)(A + m->lay.off_pf_gate); float* up = (float*)(A + m->lay.off_pf_up);
     WT* hi = (WT*)(A + m->lay.off_pf_hi); WT* lo = (WT*)(A + m->lay.off_pf_lo);
+    float* rs = (float*)(A + m->lay.off_pf_err) + 16;               // [PF_ROWS] 1/rms of the rows the planes were made from
     CK(cudaFuncSetAttribute((const void*)pf_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM));
     CK(cudaFuncSetAttribute((const void*)pf_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL));
     CK(cudaFuncSetAttribute((const void*)op_linear_kernel<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL));
@@ -1137,8 +1138,8 @@ int prefill_tc(kg_model* m, int n) {
         const int rows = n - b0 < PF_ROWS ? n - b0 : PF_ROWS;
         pf_embed_kernel<WT><<<rows, 256, 0, s>>>(D.prompt + b0, (const WT*)D.embed, c.vocab, d, h);
         auto qkv_and_append = [&](const LayerW& lw, int li) -> int {
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h, d, d, lw.g1, c.rms_eps, hi, lo);
-            int rr = pf_gemm(m, lw.wqkv, 3 * d, d, rows, qkv, nullptr);
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h, d, d, lw.g1, c.rms_eps, hi, lo, rs);
+            int rr = pf_gemm(m, lw.wqkv, 3 * d, d, rows, qkv, nullptr, rs);
             if (rr != KG_OK) return rr;
             pf_rope_append_kernel<WT><<<dim3(rows, H), 64, 0, s>>>(D, qkv, b0, (WT*)D.kcache + (size_t)li * lstride, (WT*)D.vcache + (size_t)li * lstride);
             return KG_OK;
@@ -1150,13 +1151,13 @@ int prefill_tc(kg_model* m, int n) {
             at.qkv = qkv; at.M = 0; at.pos0 = b0; at.kc = (WT*)D.kcache + (size_t)i * lstride; at.vc = (WT*)D.vcache + (size_t)i * lstride;
             at.out = attn; at.opk = nullptr;
             pf_attention_kernel<<<m->nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, at, rows);
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(attn, d, d, nullptr, 0.f, hi, lo);
-            if ((r = pf_gemm(m, lw.wo, d, d, rows, h2, h)) != KG_OK) return r;
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h2, d, d, lw.g2, c.rms_eps, hi, lo);
-            if ((r = pf_gemm(m, lw.wgate, F, d, rows, gate, nullptr)) != KG_OK) return r;
-            if ((r = pf_gemm(m, lw.wup, F, d, rows, up, nullptr)) != KG_OK) return r;
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(attn, d, d, nullptr, 0.f, hi, lo, nullptr);
+            if ((r = pf_gemm(m, lw.wo, d, d, rows, h2, h, nullptr)) != KG_OK) return r;
+            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h2, d, d, lw.g2, c.rms_eps, hi, lo, rs);
+            if ((r = pf_gemm(m, lw.wgate, F, d, rows, gate, nullptr, rs)) != KG_OK) return r;
+            if ((r = pf_gemm(m, lw.wup, F, d, rows, up, nullptr, rs)) != KG_OK) return r;
             pf_swiglu_split_kernel<<<rows, 256, 0, s>>>(gate, up, F, hi, lo);
-            if ((r = pf_gemm(m, lw.wdown, d, F, rows, h, h2)) != KG_OK) return r;
+            if ((r = pf_gemm(m, lw.wdown, d, F, rows, h, h2, nullptr)) != KG_OK) return r;
             if (i == c.exit_layer - 1 && (r = qkv_and_append(m->layers_host[L], L)) != KG_OK) return r;      // the adapter's K / V
         }
         CK(cudaGetLastError());
@@ -1182,5 +1183,34 @@ int prefill_tc(kg_model* m, int n) {
 extern "C" int kg_debug_set_prefill_mode(kg_model* m, int mode) {
     if (!m || (mode != 0 && mode != 1)) return KG_E_ARG;
     m->prefill_mode = mode;
+    return KG_OK;
+}
+
+extern "C" int kg_op_gemm(const void* W, int32_t N, int32_t K, const float* x, int32_t M, const float* resid, float* out,
+                          void* scratch, void* stream) {
+    if (!W || !x || !out || !scratch || M < 1 || N < 1 || K < 1) return KG_E_ARG;
+    if (!aligned16(W) || !aligned16(x) || !aligned16(resid) || !aligned16(out) || !aligned16(scratch)) return KG_E_ARG;
+    if (N % GM_BN || K % GM_BK) return KG_E_ARG;
+    const int rows_pad = (M + GM_BM - 1) / GM_BM * GM_BM;
+    OpScratch sc = op_layout();
+    if ((size_t)rows_pad * K * 4 > 4 * (size_t)KG_M_MAX * S_CAP * 8192) return KG_E_LIMIT;  // both planes live in the split-partial scratch
+    if (!encode_tiled_fn()) { std::snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled is not available"); return KG_E_CUDA; }
+    cudaStream_t s = (cudaStream_t)stream;
+    __nv_bfloat16* hi = (__nv_bfloat16*)((char*)scratch + sc.off_po);
+    __nv_bfloat16* lo = hi + (size_t)rows_pad * K;
+    int* err = (int*)((char*)scratch + sc.off_cnt);
+    CK(cudaMemsetAsync(err, 0, 4, s));
+    CK(cudaMemsetAsync(hi, 0, (size_t)rows_pad * K * 4, s));
+    CK(cudaFuncSetAttribute((const void*)pf_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM));
+    pf_norm_split_kernel<<<M, 256, 0, s>>>(x, K, K, nullptr, 0.f, hi, lo, nullptr);
+    CUtensorMap th, tl, tw;
+    if (!make_tmap(&th, hi, rows_pad, K) || !make_tmap(&tl, lo, rows_pad, K) || !make_tmap(&tw, W, N, K)) {
+        std::snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
+        return KG_E_CUDA;
+    }
+    GemmArgs g;
+    g.C = out; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = nullptr; g.rows = M; g.N = N; g.K = K; g.err = err;
+    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, s>>>(th, tl, tw, g);
+    CK(cudaGetLastError());
     return KG_OK;
 }

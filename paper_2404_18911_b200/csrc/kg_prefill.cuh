@@ -6,8 +6,9 @@
 // swizzle), tcgen05.mma issued by one thread with the accumulators in tensor memory, and an epilogue that reads
 // them back with tcgen05.ld.  The activations keep fp32 accuracy the same way as in the decode path: every value
 // is split into two bf16 planes, x = hi + lo, and both planes are multiplied with the bf16 weights into the same
-// fp32 accumulator.  The tensor core's fp32 accumulation rounds toward zero, which biases long chains; the k blocks
-// therefore rotate over four accumulators (all 512 tensor-memory columns) that the epilogue adds in fp32.
+// fp32 accumulator.  The tensor core's fp32 accumulation rounds toward zero, which biases long chains; every k block
+// of 64 therefore gets a fresh accumulator (four rotate through the 512 tensor-memory columns) that the epilogue
+// warps add to fp32 registers while the next blocks are being multiplied.
 //
 // Around the GEMMs sit small elementwise kernels (embedding gather, RMSNorm + split into planes, SwiGLU + split,
 // RoPE + KV append) and the tensor-core attention of the decode path run over (row block, head) items.
@@ -26,12 +27,13 @@ constexpr int GM_TILE_BYTES = GM_BM * GM_BK * 2;                       // one 12
 constexpr int GM_STAGE_BYTES = 3 * GM_TILE_BYTES;                      // A hi, A lo, W
 constexpr int GM_SMEM = GM_STAGES * GM_STAGE_BYTES + 1024 + 256;       // + alignment slack + barriers
 constexpr int GM_THREADS = 192;                                        // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr int GM_ACC = 4;                                              // rotating accumulators of 128 columns
+constexpr int GM_ACC = 4;                                              // rotating accumulators of 128 columns (= stages)
 constexpr unsigned long long GM_WAIT_CLK = 4000000000ull;              // ~2 s: a wait that runs this long gives up
 
 struct GemmArgs {
     float* C; int ldc;                  // [rows, N] fp32
-    const float* resid; int ldr;        // optional: C = resid + A W^T
+    const float* resid; int ldr;        // optional: C = resid + rowscale * A W^T
+    const float* rowscale;              // optional: one factor per row (1/rms of the row the planes were made from)
     int rows;                           // valid rows (the planes hold a multiple of 128, zero beyond)
     int N, K;                           // multiples of 128 and 64
     int* err;                           // set to 1 when a bounded wait expired
@@ -90,22 +92,26 @@ __device__ __forceinline__ bool gm_wait(unsigned long long* bar, unsigned parity
 }
 
 // ---- the GEMM ------------------------------------------------------------------------------------------------------
-// grid = (N / 128, row tiles); one 128 x 128 tile of C per CTA.
+// grid = (N / 128, row tiles); one 128 x 128 tile of C per CTA.  k block kb uses shared-memory stage kb mod 4 and
+// tensor-memory accumulator kb mod 4: its eight MMAs (four k16-steps, hi and lo plane) start a fresh accumulator, one
+// tcgen05.commit tells the producer that the stage is free and the epilogue warps that the accumulator is complete,
+// and the epilogue warps add it to their fp32 registers (round to nearest) and hand the accumulator back.  No sum
+// therefore passes through more than eight of the tensor core's truncating accumulations.
 __global__ void __launch_bounds__(GM_THREADS, 1) pf_gemm_kernel(const __grid_constant__ CUtensorMap tm_hi, const __grid_constant__ CUtensorMap tm_lo,
                                                                 const __grid_constant__ CUtensorMap tm_w, const GemmArgs g) {
     extern __shared__ __align__(128) char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     char* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);              // swizzled tiles sit on 1024-byte boundaries
-    unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + GM_STAGES * GM_STAGE_BYTES);
-    unsigned long long* empty = full + GM_STAGES;
-    unsigned long long* done = empty + GM_STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+    unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + GM_STAGES * GM_STAGE_BYTES);   // TMA -> MMA: stage filled
+    unsigned long long* mma_done = full + GM_STAGES;      // MMA -> TMA, epilogue: the k block's MMAs have completed
+    unsigned long long* acc_free = mma_done + GM_STAGES;  // epilogue -> MMA: the accumulator has been read (one arrival per warp)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + GM_ACC);
+    static_assert(GM_STAGES == GM_ACC, "a k block's stage and accumulator share one index and one completion barrier");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * GM_BN, m0 = blockIdx.y * GM_BM;
     const int nkb = g.K / GM_BK;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < GM_STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-        mbar_init(done, 1);
+        for (int i = 0; i < GM_STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&mma_done[i], 1); mbar_init(&acc_free[i], 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -122,7 +128,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) pf_gemm_kernel(const __grid_con
         // ---- TMA producer: A hi, A lo and W boxes of one k block per stage
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % GM_STAGES;
-            if (!gm_wait(&empty[s], ((unsigned)(kb / GM_STAGES) & 1u) ^ 1u, g.err)) break;
+            if (!gm_wait(&mma_done[s], ((unsigned)(kb / GM_STAGES) & 1u) ^ 1u, g.err)) break;
             const uint32_t dst = smem_u32(smem + s * GM_STAGE_BYTES), bar = smem_u32(&full[s]);
             mbar_arrive_expect_tx(&full[s], (unsigned)GM_STAGE_BYTES);
             tma_load_2d(dst, &tm_hi, kb * GM_BK, m0, bar);
@@ -130,56 +136,66 @@ __global__ void __launch_bounds__(GM_THREADS, 1) pf_gemm_kernel(const __grid_con
             tma_load_2d(dst + 2 * GM_TILE_BYTES, &tm_w, kb * GM_BK, n0, bar);
         }
     } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer: 4 k16-steps x (hi, lo) per stage into accumulator kb mod 4
+        // ---- MMA issuer
         const uint32_t idesc = umma_idesc_128(GM_BN);
-        bool ok = true;
-        for (int kb = 0; kb < nkb && ok; ++kb) {
+        for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % GM_STAGES;
-            ok = gm_wait(&full[s], (unsigned)(kb / GM_STAGES) & 1u, g.err);
-            if (!ok) break;
+            const unsigned par = (unsigned)(kb / GM_STAGES) & 1u;
+            if (!gm_wait(&acc_free[s], par ^ 1u, g.err)) break;
+            if (!gm_wait(&full[s], par, g.err)) break;
             tc_fence_after();
             const uint32_t a_hi = umma_desc_lo(smem_u32(smem + s * GM_STAGE_BYTES));
             const uint32_t a_lo = umma_desc_lo(smem_u32(smem + s * GM_STAGE_BYTES + GM_TILE_BYTES));
             const uint32_t w = umma_desc_lo(smem_u32(smem + s * GM_STAGE_BYTES + 2 * GM_TILE_BYTES));
-            const uint32_t d = tmem + (uint32_t)(kb % GM_ACC) * GM_BN;
+            const uint32_t d = tmem + (uint32_t)s * GM_BN;
 #pragma unroll
             for (int k16 = 0; k16 < GM_BK / 16; ++k16) {
-                umma_bf16(d, a_hi + 2u * k16, w + 2u * k16, idesc, (kb >= GM_ACC || k16 > 0) ? 1u : 0u);
+                umma_bf16(d, a_hi + 2u * k16, w + 2u * k16, idesc, k16 > 0 ? 1u : 0u);
                 umma_bf16(d, a_lo + 2u * k16, w + 2u * k16, idesc, 1u);
             }
-            umma_commit(&empty[s]);                      // the stage is free once these MMAs have read it
+            umma_commit(&mma_done[s]);
         }
-        umma_commit(done);
     } else if (warp >= 2) {
-        // ---- epilogue: thread = one row of the tile (tensor-memory lane), 32 columns at a time
+        // ---- epilogue: thread = one row of the tile (tensor-memory lane); the 128 columns of the row live in registers
         const int q = warp & 3;
         const int row = m0 + q * 32 + lane;
-        const int nacc = nkb < GM_ACC ? nkb : GM_ACC;
-        if (gm_wait(done, 0u, g.err)) {
+        float acc[GM_BN];
+#pragma unroll
+        for (int i = 0; i < GM_BN; ++i) acc[i] = 0.f;
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % GM_ACC;
+            ok = gm_wait(&mma_done[s], (unsigned)(kb / GM_ACC) & 1u, g.err);
+            if (!ok) break;
             tc_fence_after();
+#pragma unroll
             for (int c0 = 0; c0 < GM_BN; c0 += 32) {
-                float acc[32];
-                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
-                for (int a = 1; a < nacc; ++a) {
-                    float v[32];
-                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * GM_BN + c0), v);
+                float v[32];
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * GM_BN + c0), v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[i] += v[i];
-                }
-                if (row < g.rows) {
-                    float* dst = g.C + (size_t)row * g.ldc + n0 + c0;
-                    if (g.resid) {
-                        const float* rs = g.resid + (size_t)row * g.ldr + n0 + c0;
+                for (int i = 0; i < 32; ++i) acc[c0 + i] += v[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_free[s]);
+        }
+        if (ok && row < g.rows) {
+            float* dst = g.C + (size_t)row * g.ldc + n0;
+            if (g.rowscale) {
+                const float rsc = g.rowscale[row];
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            const float4 r4 = *reinterpret_cast<const float4*>(rs + i);
-                            acc[i] += r4.x; acc[i + 1] += r4.y; acc[i + 2] += r4.z; acc[i + 3] += r4.w;
-                        }
-                    }
+                for (int i = 0; i < GM_BN; ++i) acc[i] *= rsc;
+            }
+            if (g.resid) {
+                const float* rs = g.resid + (size_t)row * g.ldr + n0;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+                for (int i = 0; i < GM_BN; i += 4) {
+                    const float4 r4 = *reinterpret_cast<const float4*>(rs + i);
+                    acc[i] += r4.x; acc[i + 1] += r4.y; acc[i + 2] += r4.z; acc[i + 3] += r4.w;
                 }
             }
+#pragma unroll
+            for (int i = 0; i < GM_BN; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
         }
     }
     tc_fence_before();
@@ -206,12 +222,13 @@ __global__ void pf_embed_kernel(const int* toks, const WT* E, int V, int d, floa
     for (int e = threadIdx.x; e < d; e += blockDim.x) h[(size_t)r * d + e] = wt_to_float<WT>(E[(size_t)tok * d + e]);
 }
 
-// planes of RMSNorm(x[r]; gain) (gain == null: of x[r] itself); one CTA per row
-__global__ void pf_norm_split_kernel(const float* x, int ldx, int K, const float* gain, float eps, __nv_bfloat16* hi, __nv_bfloat16* lo) {
+// planes of x[r] * gain (gain == null: of x[r] itself) and, with a gain, rs[r] = 1 / rms(x[r]): the GEMM that reads the
+// planes multiplies its rows by rs afterwards, in fp32, exactly as the decode path's linear operator does (values that
+// are exact in bf16, such as embedding rows under a unit gain, then stay exact).  One CTA per row.
+__global__ void pf_norm_split_kernel(const float* x, int ldx, int K, const float* gain, float eps, __nv_bfloat16* hi, __nv_bfloat16* lo, float* rs) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const float* xr = x + (size_t)r * ldx;
-    float scale = 1.0f;
     if (gain) {
         float ss = 0.f;
         for (int k = threadIdx.x; k < K; k += blockDim.x) { const float v = xr[k]; ss += v * v; }
@@ -221,12 +238,10 @@ __global__ void pf_norm_split_kernel(const float* x, int ldx, int K, const float
         if (threadIdx.x < 32) {
             float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
             t = warp_sum(t);
-            if (threadIdx.x == 0) red[0] = rsqrtf(t / (float)K + eps);
+            if (threadIdx.x == 0) rs[r] = rsqrtf(t / (float)K + eps);
         }
-        __syncthreads();
-        scale = red[0];
     }
-    for (int k = threadIdx.x; k < K; k += blockDim.x) split_store(hi, lo, (size_t)r * K + k, gain ? (xr[k] * gain[k]) * scale : xr[k]);
+    for (int k = threadIdx.x; k < K; k += blockDim.x) split_store(hi, lo, (size_t)r * K + k, gain ? xr[k] * gain[k] : xr[k]);
 }
 
 // planes of SiLU(gate) * up

