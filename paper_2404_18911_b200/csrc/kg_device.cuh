@@ -191,10 +191,17 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// global -> shared bulk copy; bytes and both addresses are multiples of 16
-__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsigned bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// global -> shared bulk copy; bytes and both addresses are multiples of 16.  `policy` is an L2 cache policy made by
+// l2_evict_first(): weights are read once per pass, so their lines are the first to go, and what the pass re-reads
+// (activations, K/V of the draft layers, barrier words) stays in L2 while 1-65 GB of weights stream past it.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsigned bytes, unsigned long long* bar, unsigned long long policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long l2_evict_first() {
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 
 // The top bit of the grid barrier's arrival counter tells every CTA that some wait has given up: they learn it from
@@ -444,6 +451,7 @@ __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
     char* ring = c.smem + RING_OFF;
     Ctrl* ctl = c.ctl;
     int slot = c.slot; unsigned phase = c.phase; unsigned issued = c.issued;     // ring cursor, kept in registers here
+    const unsigned long long policy = l2_evict_first();
     for (int sc0 = pl.u0; sc0 < pl.u1; sc0 += pl.sc_units) {
         const int sc1 = min(pl.u1, sc0 + pl.sc_units);
         const int ngrp = (sc1 - sc0 + ST_ROWS - 1) / ST_ROWS;
@@ -460,7 +468,7 @@ __device__ __noinline__ bool lin_produce(const LinArgs& a, Ctx& c) {
                 if (!ok) { c.slot = slot; c.phase = phase; c.issued = issued; return false; }
                 if (lane == 0) mbar_arrive_expect_tx(&ctl->full[slot], (unsigned)(nvalid * len * 2));
                 __syncwarp();
-                if (lane < nvalid) bulk_g2s(ring + (size_t)slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &ctl->full[slot]);
+                if (lane < nvalid) bulk_g2s(ring + (size_t)slot * SLOT_BYTES + lane * ST_ROW_BYTES, src, (unsigned)(len * 2), &ctl->full[slot], policy);
                 issued++;
                 if (++slot == RING) { slot = 0; phase ^= 1u; }
             }
@@ -670,23 +678,29 @@ __device__ __noinline__ void lin_consume(const LinArgs& a, Ctx& c) {
                 if (ok) {
                     // ldmatrix x4: matrices 0, 2 = rows 0-7 (first stage), 1, 3 = rows 8-15 (second stage); k halves 0-7 | 8-15
                     const uint32_t a_base = smem_u32(ring + (size_t)((lane & 8) ? slot_b : slot_a) * SLOT_BYTES) + a_lane;
+                    // the weight fragments are fetched PD steps ahead of the MMA that uses them (the loads and the MMAs
+                    // issue in program order, so a load right before its MMA would expose its latency at every step);
+                    // loads past the phase's last step stay inside the slot and are never used
+                    constexpr int PD = V == 4 ? 4 : 2;
+                    unsigned af[PD][4];
+#pragma unroll
+                    for (int s = 0; s < PD; ++s) ldmatrix_x4(af[s], a_base + (uint32_t)s * 32u);
 #pragma unroll
                     for (int s = 0; s < NS; ++s) {
                         if (warp * NS + s < nsteps) {
-                            unsigned af[4];
-                            ldmatrix_x4(af, a_base + (uint32_t)s * 32u);
                             if (V == 4) {
-                                mma_bf16_16816(acc[s & 3], af, fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[s & 3], af[s % PD], fr[s][0], fr[s][1]);
                             } else if (V == 8) {
-                                mma_bf16_16816(acc[(s & 1) * 2], af, fr[s][0], fr[s][1]);
-                                mma_bf16_16816(acc[(s & 1) * 2 + 1], af, fr[s][2], fr[s][3]);
+                                mma_bf16_16816(acc[(s & 1) * 2], af[s % PD], fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[(s & 1) * 2 + 1], af[s % PD], fr[s][2], fr[s][3]);
                             } else {
-                                mma_bf16_16816(acc[0], af, fr[s][0], fr[s][1]);
-                                mma_bf16_16816(acc[1], af, fr[s][2], fr[s][3]);
-                                mma_bf16_16816(acc[2], af, fr[s][FR - 4], fr[s][FR - 3]);
-                                mma_bf16_16816(acc[3], af, fr[s][FR - 2], fr[s][FR - 1]);
+                                mma_bf16_16816(acc[0], af[s % PD], fr[s][0], fr[s][1]);
+                                mma_bf16_16816(acc[1], af[s % PD], fr[s][2], fr[s][3]);
+                                mma_bf16_16816(acc[2], af[s % PD], fr[s][FR - 4], fr[s][FR - 3]);
+                                mma_bf16_16816(acc[3], af[s % PD], fr[s][FR - 2], fr[s][FR - 1]);
                             }
                         }
+                        if (s + PD < NS) ldmatrix_x4(af[s % PD], a_base + (uint32_t)(s + PD) * 32u);
                     }
                 }
                 __syncwarp();
