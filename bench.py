@@ -288,6 +288,8 @@ def run_kangaroo(args):
         shape = shape.with_(n_prompt=args.n_prompt)
     if args.layers:
         shape = shape.with_(n_layers=args.layers, name=f"{shape.name}-{args.layers}layers")
+    if shape.n_prompt + shape.n_gen + shape.gamma + 8 > shape.max_seq:
+        shape = shape.with_(max_seq=shape.n_prompt + shape.n_gen + shape.gamma + 8)
     mode = binding.STOP_DROP if args.stop == "drop" else binding.STOP_KEEP
     model = binding.KangarooModel(shape, device=f"cuda:{local_rank}")
     prompt_np = ki.make_prompt(shape)

@@ -113,7 +113,8 @@ struct Layout {
 // The tensor-core prompt pass needs bf16 weights, a head_dim the tensor-core attention knows, and matrix sides that
 // are whole tiles: N a multiple of 128, K a multiple of 64.
 bool prefill_tc_shape(const kg_config* c) {
-    return c->dtype == KG_BF16 && (c->head_dim == 64 || c->head_dim == 128) && c->d_model % 128 == 0 && c->d_ffn % 128 == 0;
+    return c->dtype == KG_BF16 && (c->head_dim == 64 || c->head_dim == 128) && c->d_model % 128 == 0 && c->d_ffn % 128 == 0 &&
+           c->d_model <= PF_EW_THREADS * 4 * PF_NORM_V;      // the norm kernel keeps a row in registers
 }
 
 bool valid_config(const kg_config* c) {
@@ -1074,20 +1075,19 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K) {
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-__global__ void __launch_bounds__(BLOCK_THREADS, 1) pf_attention_kernel(const __grid_constant__ Dev D, AttArgs a, int nrows) {
+// launched with the consumer warps only (no copy warp: nothing is streamed), which leaves 255 registers per thread
+__global__ void __launch_bounds__(NTHREADS, 1) pf_attention_kernel(const __grid_constant__ Dev D, AttArgs a, int nrows) {
     extern __shared__ __align__(128) char smem[];
     Ctx& c = ctx_init(smem, nullptr, nullptr, false);
-    if (!c.producer) {
-        if (D.dm.hd == 128) attention_prefill<128>(D, a, c, nrows);
-        else attention_prefill<64>(D, a, c, nrows);
-    }
+    if (D.dm.hd == 128) attention_prefill<128>(D, a, c, nrows);
+    else attention_prefill<64>(D, a, c, nrows);
 }
 
-// x_0 from the per-CTA LM-head partials; the sequence state after a prompt of n tokens
+// x_0 from the per-CTA LM-head partials; the sequence state after a prompt of n tokens (one warp)
 __global__ void pf_finish_kernel(const float4* part, int nctas, State* st, int* out_tokens, int n, const int* gemm_err) {
+    int tok; float p;
+    head_final_warp(part, nctas, 0, tok, p);
     if (threadIdx.x == 0) {
-        int tok; float p;
-        head_final(part, nctas, 0, tok, p);
         if (*gemm_err) { atomicCAS(&st->status, 0, ST_TIMEOUT); st->timeout_where = 60; }      // a wait inside a GEMM gave up
         st->P = n; st->len_A = n; st->x0 = tok; st->pending = 0; st->total = 1; st->rounds = 0;
         out_tokens[0] = tok;
@@ -1098,18 +1098,20 @@ bool prefill_tc_ok(const kg_model* m, int n) {
     return m->prefill_mode == 0 && m->dev.dm.stream != 0 && prefill_tc_shape(&m->cfg) && n >= 2 * KG_M_MAX && encode_tiled_fn() != nullptr;
 }
 
-// C[rows, N] = (resid) + planes[rows, K] W[N, K]^T
-int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const float* resid, const float* rowscale) {
+// C[rows, N] = (resid) + rowscale * planes[rows, K] W[N, K]^T; with W2: also C2 = rowscale * planes W2^T in the same launch
+int pf_gemm(kg_model* m, const void* W, int N, int K, int rows, float* C, const float* resid, const float* rowscale,
+            const void* W2 = nullptr, float* C2 = nullptr) {
     char* A = m->arena;
     const int rows_pad = (rows + GM_BM - 1) / GM_BM * GM_BM;
-    CUtensorMap th, tl, tw;
-    if (!make_tmap(&th, A + m->lay.off_pf_hi, rows_pad, K) || !make_tmap(&tl, A + m->lay.off_pf_lo, rows_pad, K) || !make_tmap(&tw, W, N, K)) {
+    CUtensorMap th, tl, tw, tw2;
+    if (!make_tmap(&th, A + m->lay.off_pf_hi, rows_pad, K) || !make_tmap(&tl, A + m->lay.off_pf_lo, rows_pad, K) || !make_tmap(&tw, W, N, K) ||
+        !make_tmap(&tw2, W2 ? W2 : W, N, K)) {
         std::snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
         return KG_E_CUDA;
     }
     GemmArgs g;
-    g.C = C; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = rowscale; g.rows = rows; g.N = N; g.K = K; g.err = (int*)(A + m->lay.off_pf_err);
-    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, m->stream>>>(th, tl, tw, g);
+    g.C = C; g.C2 = C2; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = rowscale; g.rows = rows; g.N = N; g.K = K; g.err = (int*)(A + m->lay.off_pf_err);
+    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM, W2 ? 2 : 1), GM_THREADS, GM_SMEM, m->stream>>>(th, tl, tw, tw2, g);
     CK(cudaGetLastError());
     return KG_OK;
 }
@@ -1138,7 +1140,7 @@ int prefill_tc(kg_model* m, int n) {
         const int rows = n - b0 < PF_ROWS ? n - b0 : PF_ROWS;
         pf_embed_kernel<WT><<<rows, 256, 0, s>>>(D.prompt + b0, (const WT*)D.embed, c.vocab, d, h);
         auto qkv_and_append = [&](const LayerW& lw, int li) -> int {
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h, d, d, lw.g1, c.rms_eps, hi, lo, rs);
+            pf_norm_split_kernel<<<rows, PF_EW_THREADS, 0, s>>>(h, d, d, lw.g1, c.rms_eps, hi, lo, rs);
             int rr = pf_gemm(m, lw.wqkv, 3 * d, d, rows, qkv, nullptr, rs);
             if (rr != KG_OK) return rr;
             pf_rope_append_kernel<WT><<<dim3(rows, H), 64, 0, s>>>(D, qkv, b0, (WT*)D.kcache + (size_t)li * lstride, (WT*)D.vcache + (size_t)li * lstride);
@@ -1150,13 +1152,12 @@ int prefill_tc(kg_model* m, int n) {
             AttArgs at;
             at.qkv = qkv; at.M = 0; at.pos0 = b0; at.kc = (WT*)D.kcache + (size_t)i * lstride; at.vc = (WT*)D.vcache + (size_t)i * lstride;
             at.out = attn; at.opk = nullptr;
-            pf_attention_kernel<<<m->nctas, BLOCK_THREADS, SMEM_TOTAL, s>>>(D, at, rows);
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(attn, d, d, nullptr, 0.f, hi, lo, nullptr);
+            pf_attention_kernel<<<m->nctas, NTHREADS, SMEM_TOTAL, s>>>(D, at, rows);
+            pf_split_kernel<<<dim3(rows, (d / 4 + PF_EW_THREADS - 1) / PF_EW_THREADS), PF_EW_THREADS, 0, s>>>(attn, d, d, hi, lo);
             if ((r = pf_gemm(m, lw.wo, d, d, rows, h2, h, nullptr)) != KG_OK) return r;
-            pf_norm_split_kernel<<<rows, 256, 0, s>>>(h2, d, d, lw.g2, c.rms_eps, hi, lo, rs);
-            if ((r = pf_gemm(m, lw.wgate, F, d, rows, gate, nullptr, rs)) != KG_OK) return r;
-            if ((r = pf_gemm(m, lw.wup, F, d, rows, up, nullptr, rs)) != KG_OK) return r;
-            pf_swiglu_split_kernel<<<rows, 256, 0, s>>>(gate, up, F, hi, lo);
+            pf_norm_split_kernel<<<rows, PF_EW_THREADS, 0, s>>>(h2, d, d, lw.g2, c.rms_eps, hi, lo, rs);
+            if ((r = pf_gemm(m, lw.wgate, F, d, rows, gate, nullptr, rs, lw.wup, up)) != KG_OK) return r;
+            pf_swiglu_split_kernel<<<dim3(rows, (F / 4 + PF_EW_THREADS - 1) / PF_EW_THREADS), PF_EW_THREADS, 0, s>>>(gate, up, F, hi, lo);
             if ((r = pf_gemm(m, lw.wdown, d, F, rows, h, h2, nullptr)) != KG_OK) return r;
             if (i == c.exit_layer - 1 && (r = qkv_and_append(m->layers_host[L], L)) != KG_OK) return r;      // the adapter's K / V
         }
@@ -1202,15 +1203,15 @@ extern "C" int kg_op_gemm(const void* W, int32_t N, int32_t K, const float* x, i
     CK(cudaMemsetAsync(err, 0, 4, s));
     CK(cudaMemsetAsync(hi, 0, (size_t)rows_pad * K * 4, s));
     CK(cudaFuncSetAttribute((const void*)pf_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM));
-    pf_norm_split_kernel<<<M, 256, 0, s>>>(x, K, K, nullptr, 0.f, hi, lo, nullptr);
+    pf_split_kernel<<<dim3(M, (K / 4 + PF_EW_THREADS - 1) / PF_EW_THREADS), PF_EW_THREADS, 0, s>>>(x, K, K, hi, lo);
     CUtensorMap th, tl, tw;
     if (!make_tmap(&th, hi, rows_pad, K) || !make_tmap(&tl, lo, rows_pad, K) || !make_tmap(&tw, W, N, K)) {
         std::snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
         return KG_E_CUDA;
     }
     GemmArgs g;
-    g.C = out; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = nullptr; g.rows = M; g.N = N; g.K = K; g.err = err;
-    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, s>>>(th, tl, tw, g);
+    g.C = out; g.C2 = nullptr; g.ldc = N; g.resid = resid; g.ldr = N; g.rowscale = nullptr; g.rows = M; g.N = N; g.K = K; g.err = err;
+    pf_gemm_kernel<<<dim3(N / GM_BN, rows_pad / GM_BM), GM_THREADS, GM_SMEM, s>>>(th, tl, tw, tw, g);
     CK(cudaGetLastError());
     return KG_OK;
 }

@@ -1571,7 +1571,8 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
     };
     // One register set for K and V (a second one would not fit: the register allocation is shared with the
     // linear operators).  A tile therefore costs a memory latency; the split count above keeps the run of
-    // tiles per unit short, and the other units and CTAs keep the memory system busy meanwhile.
+    // tiles per unit short, and the other units and CTAs keep the memory system busy meanwhile.  (In the prompt
+    // pass, where a unit walks over hundreds of tiles, requesting the next tile early was measured: 2 % slower.)
     AttK k0;
     AttV v0;
     while (tile < tend) {
