@@ -1363,7 +1363,7 @@ template <int HD> struct AttSm {
     static constexpr int QS = HD * 2 + 64;                      // bytes per Q row (padded: two rows per shared-memory phase)
     static constexpr int Q_BYTES = 2 * M_MAX * QS;              // hi plane, lo plane
     static constexpr int MB_OFF = (Q_BYTES + 15) / 16 * 16;     // merge buffer [units][ATT_RB][ATT_MB_STRIDE] floats; while the
-                                                                // tiles run, the pairs' score exchange [4][2][2][32] float4
+                                                                // tiles run, the pairs' score exchange [4][2][1 or 2][2][32] float4
 };
 
 // Page-table entries of a window of 32 pages, one per lane; a lane asks for the page of a key by shuffle.
@@ -1481,7 +1481,7 @@ __device__ __forceinline__ void att_accumulate(const AttV& tv, AttAcc& ac, const
 // One work item of the tensor-core attention: head hh, split s of S (chunk_tiles tiles each) of the keys 0 .. pos0 + M - 1
 // for the rows of `a`.  append: this pass's K / V rows are rotated, rounded and written to the cache by the item whose
 // key range holds them (false: they are in the cache already).
-template <int HD>
+template <int HD, bool DUAL = false>
 __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c, int hh, int s, int S, int chunk_tiles, bool append) {
     typedef __nv_bfloat16 WT;
     constexpr int NSPLIT = HD / ATT_DW;               // warps per unit: 1 (head_dim 64) or 2 (head_dim 128)
@@ -1495,7 +1495,10 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
     const int T = pos0 + M;
     const int ntiles_all = (T + ATT_TK - 1) / ATT_TK;
     const int R = (M + 7) >> 3;                       // row groups of 8
-    const int nw = NUNITS / R;                        // units that share the tiles of an item (a power of two)
+    // DUAL (prompt pass, two row groups): every unit works on both row groups of its tiles, two independent chains of
+    // dependent instructions side by side; else a unit owns one row group
+    constexpr int NRG = DUAL ? 2 : 1;
+    const int nw = DUAL ? NUNITS : NUNITS / R;        // units that share the tiles of an item (a power of two)
     const int tpw = (chunk_tiles + nw - 1) / nw;
     const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;      // 1/sqrt(hd) and log2(e)
     WT* kc = reinterpret_cast<WT*>(a.kc);
@@ -1503,7 +1506,7 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
     unsigned char* qs = reinterpret_cast<unsigned char*>(c.smem + WORK_OFF);
     float* mb = reinterpret_cast<float*>(c.smem + WORK_OFF + AttSm<HD>::MB_OFF);
     const int unit = warp / NSPLIT, hsel = warp % NSPLIT, dof = hsel * ATT_DW;
-    const int rg = unit % R, tlane = unit / R;
+    const int rg = DUAL ? 0 : unit % R, tlane = DUAL ? unit : unit / R;
     const int row0 = rg * 8;
     const uint32_t qw = smem_u32(qs) + (uint32_t)(dof * 2);
     // rows >= M of the row groups in use are zero in both planes
@@ -1539,10 +1542,13 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
             vc[base + e + half] = __float2bfloat16_rn(v2);
         }
     }
-    AttAcc ac;
+    AttAcc ac[NRG];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { ac.o[e][0] = ac.o[e][1] = ac.o[e][2] = ac.o[e][3] = 0.f; }
-    ac.m[0] = ac.m[1] = -INFINITY; ac.l[0] = ac.l[1] = 0.f;
+    for (int r = 0; r < NRG; ++r) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { ac[r].o[e][0] = ac[r].o[e][1] = ac[r].o[e][2] = ac[r].o[e][3] = 0.f; }
+        ac[r].m[0] = ac[r].m[1] = -INFINITY; ac[r].l[0] = ac[r].l[1] = 0.f;
+    }
     // this unit's tiles: a contiguous run, so that one window of page-table entries serves many of them
     int tile = tb + tlane * tpw;
     const int tend = min(te, tile + tpw);
@@ -1554,20 +1560,27 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
         if ((key1 >> psh) - pw.first >= 32) pw.load(D.page_table, D.dm.n_pages, key0 >> psh);
         att_load<HD>(tk, tv, kc, vc, pw, H, hh, dof, psh, psm, key0, T - 1, D.dm.n_phys, D.st);
     };
-    AttP pp;
+    AttP pp[NRG];
     auto step = [&](const AttK& tk, const AttV& tv, int ti) {
-        float sc[4];
-        att_scores<QS>(tk, sc, qw, row0);
+        float sc[NRG][4];
+#pragma unroll
+        for (int r = 0; r < NRG; ++r) att_scores<QS>(tk, sc[r], qw, row0 + 8 * r);
         if constexpr (NSPLIT == 2) {
             // the pair's halves of the dot products meet in shared memory (two buffers, used alternately)
-            float4* xb = reinterpret_cast<float4*>(mb) + (size_t)((unit * 2 + (ti & 1)) * 2) * 32;
-            xb[hsel * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+            float4* xb = reinterpret_cast<float4*>(mb) + (size_t)((unit * 2 + (ti & 1)) * NRG * 2) * 32;
+#pragma unroll
+            for (int r = 0; r < NRG; ++r) xb[(r * 2 + hsel) * 32 + lane] = make_float4(sc[r][0], sc[r][1], sc[r][2], sc[r][3]);
             pair_sync(unit);
-            const float4 ot = xb[(hsel ^ 1) * 32 + lane];
-            sc[0] += ot.x; sc[1] += ot.y; sc[2] += ot.z; sc[3] += ot.w;
+#pragma unroll
+            for (int r = 0; r < NRG; ++r) {
+                const float4 ot = xb[(r * 2 + (hsel ^ 1)) * 32 + lane];
+                sc[r][0] += ot.x; sc[r][1] += ot.y; sc[r][2] += ot.z; sc[r][3] += ot.w;
+            }
         }
-        att_softmax(sc, ac, pp, row0, ti * ATT_TK, ke, pos0);
-        att_accumulate(tv, ac, pp);
+#pragma unroll
+        for (int r = 0; r < NRG; ++r) att_softmax(sc[r], ac[r], pp[r], row0 + 8 * r, ti * ATT_TK, ke, pos0);
+#pragma unroll
+        for (int r = 0; r < NRG; ++r) att_accumulate(tv, ac[r], pp[r]);
     };
     // One register set for K and V (a second one would not fit: the register allocation is shared with the
     // linear operators).  A tile therefore costs a memory latency; the split count above keeps the run of
@@ -1582,26 +1595,32 @@ __device__ __forceinline__ void att_item(const Dev& D, const AttArgs& a, Ctx& c,
     }
     // the row sums: lanes that share rows add their shares in a fixed order
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 4);
-        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 8);
-        ac.l[r] += __shfl_xor_sync(0xffffffffu, ac.l[r], 16);
+    for (int q = 0; q < NRG; ++q) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            ac[q].l[r] += __shfl_xor_sync(0xffffffffu, ac[q].l[r], 4);
+            ac[q].l[r] += __shfl_xor_sync(0xffffffffu, ac[q].l[r], 8);
+            ac[q].l[r] += __shfl_xor_sync(0xffffffffu, ac[q].l[r], 16);
+        }
     }
     if constexpr (NSPLIT == 2) cta_sync();          // the merge buffer lies over the pairs' exchange buffers
     // merge the units of a row group through shared memory, four rows at a time
-    for (int rb = 0; rb * ATT_RB < M; ++rb) {
+#pragma unroll
+    for (int rb = 0; rb < M_MAX / ATT_RB; ++rb) {
+        if (rb * ATT_RB >= M) break;
         const int nr = min(ATT_RB, M - rb * ATT_RB);
-        if (rg == (rb >> 1) && (t >> 1) == (rb & 1)) {
+        const AttAcc& aa = ac[NRG == 2 ? (rb >> 1) : 0];
+        if ((DUAL || rg == (rb >> 1)) && (t >> 1) == (rb & 1)) {
             const int rl = 2 * (t & 1);
             float* r0 = mb + ((size_t)tlane * ATT_RB + rl) * ATT_MB_STRIDE;
             float* r1 = r0 + ATT_MB_STRIDE;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int dd = dof + 8 * g + 2 * e;
-                *reinterpret_cast<float2*>(r0 + dd) = make_float2(ac.o[e][0], ac.o[e][2]);
-                *reinterpret_cast<float2*>(r1 + dd) = make_float2(ac.o[e][1], ac.o[e][3]);
+                *reinterpret_cast<float2*>(r0 + dd) = make_float2(aa.o[e][0], aa.o[e][2]);
+                *reinterpret_cast<float2*>(r1 + dd) = make_float2(aa.o[e][1], aa.o[e][3]);
             }
-            if (g == 0 && hsel == 0) { r0[HD_MAX] = ac.m[0]; r0[HD_MAX + 1] = ac.l[0]; r1[HD_MAX] = ac.m[1]; r1[HD_MAX + 1] = ac.l[1]; }
+            if (g == 0 && hsel == 0) { r0[HD_MAX] = aa.m[0]; r0[HD_MAX + 1] = aa.l[0]; r1[HD_MAX] = aa.m[1]; r1[HD_MAX + 1] = aa.l[1]; }
         }
         cta_sync();
         for (int idx = tid; idx < nr * HD; idx += NTHREADS) {
@@ -1693,10 +1712,13 @@ __device__ __noinline__ void attention_prefill(const Dev& D, const AttArgs& a, C
         b.opk = nullptr;
         b.M = min(M_MAX, nrows - rb * M_MAX);
         b.pos0 = a.pos0 + rb * M_MAX;
-        att_item<HD>(D, b, c, hh, 0, 1, (b.pos0 + b.M + ATT_TK - 1) / ATT_TK, false);
+        // full blocks of 16 rows: both row groups in every unit; a shorter last block: the decode path's split
+        if (b.M > 8) att_item<HD, true>(D, b, c, hh, 0, 1, (b.pos0 + b.M + ATT_TK - 1) / ATT_TK, false);
+        else att_item<HD, false>(D, b, c, hh, 0, 1, (b.pos0 + b.M + ATT_TK - 1) / ATT_TK, false);
     }
 }
 static_assert(AttSm<HD_MAX>::MB_OFF + NWARPS * ATT_RB * ATT_MB_STRIDE * 4 <= WORK_BYTES, "tensor-core attention buffers do not fit in the work area");
+static_assert(4 * 2 * 2 * 2 * 32 * 16 <= NWARPS * ATT_RB * ATT_MB_STRIDE * 4, "the score exchange of two row groups does not fit in the merge buffer");
 
 template <typename WT>
 __device__ __forceinline__ void attention_op(const Dev& D, const AttArgs* sa, Ctx& c) {
