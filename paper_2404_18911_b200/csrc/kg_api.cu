@@ -294,7 +294,7 @@ static int launch_program(kg_model* m, const Program& pg) {
     p.skip_arrival = m->skip_arrival;
     m->skip_arrival = 0;
     void* args[] = {(void*)&m->dev, (void*)&p};
-    CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(BLOCK_THREADS), args, m->smem, m->stream));
+    CK(cudaLaunchCooperativeKernel((const void*)kg_persistent_kernel<WT>, dim3(m->nctas), dim3(DECODE_THREADS), args, m->smem, m->stream));
     return KG_OK;
 }
 static int launch(kg_model* m, const Program& pg) {
@@ -388,7 +388,18 @@ extern "C" int kg_init_model(const kg_config* cfg, const kg_weights* w, void* ar
     const void* kfn = bf ? (const void*)kg_persistent_kernel<__nv_bfloat16> : (const void*)kg_persistent_kernel<float>;
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m->smem) != cudaSuccess) { delete m; return KG_E_CUDA; }
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kfn, BLOCK_THREADS, m->smem) != cudaSuccess || occ < 1) { delete m; return KG_E_CUDA; }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kfn, DECODE_THREADS, m->smem) != cudaSuccess || occ < 1) { delete m; return KG_E_CUDA; }
+    {
+        // the kernel's warpgroups re-divide the registers the launch gives the CTA; a budget beyond that pool would block
+        // the kernel at its first instruction, so the launch allocation is checked here, once, and never assumed
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, kfn) != cudaSuccess) { delete m; return KG_E_CUDA; }
+        if ((long long)fa.numRegs * DECODE_THREADS < (long long)NTHREADS * CONSUMER_REGS + 128LL * PRODUCER_REGS) {
+            std::snprintf(g_cuda_err, sizeof(g_cuda_err), "decode kernel compiled with %d registers per thread: too few for its register budgets", fa.numRegs);
+            delete m;
+            return KG_E_INTERNAL;
+        }
+    }
 
     Dev& D = m->dev;
     std::memset(&D, 0, sizeof(D));

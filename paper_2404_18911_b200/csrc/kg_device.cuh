@@ -25,6 +25,15 @@ constexpr int M_MAX = 16;          // rows per pass
 constexpr int NTHREADS = 256;      // consumer threads per CTA
 constexpr int NWARPS = NTHREADS / 32;
 constexpr int BLOCK_THREADS = NTHREADS + 32;   // + the producer warp (warp index NWARPS)
+// The decode kernel is launched with a whole warpgroup behind the consumers (warp NWARPS is the producer, the other
+// three leave at once): registers are handed out per warpgroup, and the producer's warpgroup gives most of its share
+// to the two consumer warpgroups at kernel start (setmaxnreg).  The pool is what the launch allocated: 384 threads x
+// 168 registers = 64512; a request beyond it would block forever, so the budgets below are checked against it.
+constexpr int DECODE_THREADS = NTHREADS + 128;
+constexpr int LAUNCH_REGS = 168;                  // 65536 / 384, rounded down to the allocation unit of 8
+constexpr int CONSUMER_REGS = 216, PRODUCER_REGS = 56;
+static_assert(NTHREADS * CONSUMER_REGS + 128 * PRODUCER_REGS <= DECODE_THREADS * LAUNCH_REGS, "register budgets exceed the CTA's pool");
+static_assert(DECODE_THREADS * (LAUNCH_REGS + 8) > 65536, "LAUNCH_REGS is not what a launch of DECODE_THREADS threads gets");
 constexpr int S_CAP = 16;          // most KV splits per head
 constexpr int HD_MAX = 128;
 
@@ -920,13 +929,7 @@ __device__ __noinline__ void lin_simple(const LinArgs& a, Ctx& c) {
 // rows exist wherever they are read).  Consumers return after their part; whether the grid must stop
 // is learnt at the next grid barrier.  The producer returns false when one of its waits gave up.
 template <typename WT>
-__device__ __forceinline__ bool linear_op(const LinArgs* sa, Ctx& c, bool stream, bool publish) {
-    // sa points into this role's operator table in shared memory; publish: the table was written just before
-    if (c.producer) {
-        if (!stream) return true;
-        if (publish) __syncwarp();
-        return lin_produce(*sa, c);
-    }
+__device__ __forceinline__ bool linear_consumer(const LinArgs* sa, Ctx& c, bool stream, bool publish) {
     if (publish) cta_sync();
     if (stream) {
         if (sa->M <= 4) lin_consume<4>(*sa, c); else if (sa->M <= 8) lin_consume<8>(*sa, c); else lin_consume<16>(*sa, c);
@@ -934,6 +937,16 @@ __device__ __forceinline__ bool linear_op(const LinArgs* sa, Ctx& c, bool stream
         lin_simple<WT>(*sa, c);
     }
     return true;
+}
+__device__ __forceinline__ bool linear_producer(const LinArgs* sa, Ctx& c, bool stream, bool publish) {
+    if (!stream) return true;
+    if (publish) __syncwarp();
+    return lin_produce(*sa, c);
+}
+template <typename WT>
+__device__ __forceinline__ bool linear_op(const LinArgs* sa, Ctx& c, bool stream, bool publish) {
+    // sa points into this role's operator table in shared memory; publish: the table was written just before
+    return c.producer ? linear_producer(sa, c, stream, publish) : linear_consumer<WT>(sa, c, stream, publish);
 }
 
 // Merge the per-CTA head partials of row m (identical result in every CTA: fixed order).

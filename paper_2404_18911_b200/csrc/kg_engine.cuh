@@ -33,7 +33,9 @@ struct Program {
 struct ActIn { const float* x; const unsigned char* pk; const float* ssq; };
 struct ActOut { float* x; PkOut pk[2]; float* ssq; };
 
-template <typename WT>
+// PROD: the instruction stream of the producer warp (it only issues weight copies and follows the control flow) or of
+// the consumer warps; the two are compiled apart because they run with different register budgets.
+template <typename WT, bool PROD>
 struct Engine {
     const Dev& D;
     Ctx& c;
@@ -43,15 +45,18 @@ struct Engine {
 
     // ---- leaf operations: what a thread does depends on its role -------------------------------
     __device__ __forceinline__ bool streamed() const { return D.dm.stream != 0 && pg.force_simple == 0; }
-    __device__ __forceinline__ bool sync(int where) { return c.producer ? true : grid_sync(c, where); }
+    __device__ __forceinline__ bool sync(int where) { if constexpr (PROD) return true; else return grid_sync(c, where); }
     // this role's operator table in shared memory, and the one thread of the role that fills it
     __device__ __forceinline__ OpTable* table() const {
-        if (c.producer) __syncwarp();        // the lanes have left the previous operator before lane 0 rewrites the table
-        return reinterpret_cast<OpTable*>(c.producer ? c.ctl->tab_prod : c.ctl->tab_cons);
+        if constexpr (PROD) __syncwarp();    // the lanes have left the previous operator before lane 0 rewrites the table
+        return reinterpret_cast<OpTable*>(PROD ? c.ctl->tab_prod : c.ctl->tab_cons);
     }
-    __device__ __forceinline__ bool writer() const { return c.producer ? (threadIdx.x & 31) == 0 : threadIdx.x == 0; }
-    __device__ __forceinline__ bool linear(const LinArgs* a, bool publish) { return linear_op<WT>(a, c, streamed(), publish); }
-    __device__ __forceinline__ void attention(const AttArgs* at) { if (!c.producer) attention_op<WT>(D, at, c); }
+    __device__ __forceinline__ bool writer() const { return PROD ? (threadIdx.x & 31) == 0 : threadIdx.x == 0; }
+    __device__ __forceinline__ bool linear(const LinArgs* a, bool publish) {
+        if constexpr (PROD) return linear_producer(a, c, streamed(), publish);
+        else return linear_consumer<WT>(a, c, streamed(), publish);
+    }
+    __device__ __forceinline__ void attention(const AttArgs* at) { if constexpr (!PROD) attention_op<WT>(D, at, c); }
 
     __device__ size_t cache_layer_stride() const {
         return (size_t)D.dm.n_pages * D.dm.H * D.dm.page_size * D.dm.hd;
@@ -71,7 +76,7 @@ struct Engine {
 
     // h[i] = E[token_i]; packed for layer 0
     __device__ void embed_rows(const int* toks_global, int tok_single, int M) {
-        if (c.producer) return;
+        if constexpr (PROD) return;
         const int d = D.dm.d;
         const WT* E = reinterpret_cast<const WT*>(D.embed);
         if (!streamed()) {
@@ -187,7 +192,7 @@ struct Engine {
             a.logits_dbg = dm.debug ? dbg : nullptr; a.ld_dbg = dm.V;
         }
         if (!linear(&t->lin[0], true)) return false;
-        if (c.producer) {
+        if constexpr (PROD) {
             // held back here until the consumers have the result
             int ok = 1;
             const unsigned mp = c.mail_phase;
@@ -294,7 +299,7 @@ struct Engine {
         while (k < n_d && dtok[k] == t[k]) ++k;
         const int newP = P + k + 1;
         if (len_A > newP) len_A = newP;
-        if (len_A < newP && !c.producer) {
+        if (len_A < newP && !PROD) {
             // the adapter has not seen f[k] (k == n_d): keep it as the feature of position newP-1 (slot 0)
             const int gtid = c.cta * NTHREADS + threadIdx.x, gn = c.nctas * NTHREADS;
             const float* src = D.feat + (size_t)(1 + k) * dm.d;
@@ -384,19 +389,29 @@ struct Engine {
 
     __device__ void run() {
         // the plain path streams nothing: its producer warp has no part in the launch
-        if (c.producer && !streamed()) return;
+        if (PROD && !streamed()) return;
         load_state();
         const bool ok = run_program();
-        if (!ok && c.producer) ring_drain(c);
+        if (!ok && PROD) ring_drain(c);
     }
 };
 
 template <typename WT>
-__global__ void __launch_bounds__(BLOCK_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
+__global__ void __launch_bounds__(DECODE_THREADS, 1) kg_persistent_kernel(const __grid_constant__ Dev D, const Program pg) {
     extern __shared__ __align__(128) char smem[];
     Ctx& c = ctx_init(smem, D.st, D.bar, true, pg.wait_clk, pg.skip_arrival);
-    Engine<WT> eng(D, c, pg);
-    eng.run();
+    if (threadIdx.x >= NTHREADS) {
+        // the producer's warpgroup: keeps what the copy loop needs and returns the rest of its registers
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PRODUCER_REGS));
+        if (threadIdx.x < BLOCK_THREADS) {
+            Engine<WT, true> eng(D, c, pg);
+            eng.run();
+        }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(CONSUMER_REGS));
+        Engine<WT, false> eng(D, c, pg);
+        eng.run();
+    }
 }
 
 }  // namespace kg
